@@ -30,7 +30,13 @@
  *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*, NULL = the
  *     legacy default stream) and return without synchronising.
  *   - Return value: VT_ATTN_OK or a negative VT_ATTN_ERR_* code.  Nothing throws.
- *     On an error return no kernel has been launched.
+ *     On an argument, shape or workspace error nothing has been launched.  After
+ *     VT_ATTN_ERR_CUDA (a launch or a driver call failed part-way through an entry point
+ *     that enqueues several kernels) the outputs are undefined.
+ *   - Threads: calls from different host threads are safe on different streams.  The
+ *     *_host entry points serialise their enqueueing inside the library (one call at a
+ *     time forks onto the library's two streams and joins back), and two such calls
+ *     that are in flight together on one device must not share a staging area.
  *   - Supported: D a multiple of 8 in [8, 128]; in the forward entry points that take
  *     [B, H, S, D] tensors (vt_attn_fwd, vt_attn_fwd_f16, vt_attn_fwd_splitkv) and the merge
  *     entry points up to 256.  The kernels are built for 64, 128 and (forward) 256 columns;
@@ -277,7 +283,9 @@ int vt_attn_fwd_splitkv_plan(int B, int Hq, int Hkv, int Sq, int Sk, int D, int 
  * group share a tile (Hq / Hkv * max_sq <= 128), are planned from the longest sequence
  * (vt_attn_fwd_splitkv_plan(n_seqs, Hq, Hkv, max_sq, max_sk, D, n_splits, ...) tells); every
  * sequence's own keys are then cut into that many chunks.  A sequence
- * without queries costs nothing; one without keys (or whose rows see none) gets O = 0, LSE = -inf.
+ * without queries costs nothing; one without keys (or whose rows see none) gets O = 0, LSE = -inf,
+ * and so do the query tokens of a sequence longer than max_sq (vt_attn_fwd_varlen leaves those
+ * untouched; pass a max_sq that covers the longest sequence).
  * workspace: device memory of at least vt_attn_fwd_splitkv_varlen_workspace_bytes(...) bytes,
  * 256-byte aligned, contents undefined afterwards.  bfloat16; D a multiple of 8 in [8, 128].
  */
@@ -353,7 +361,8 @@ size_t vt_attn_host_staging_bytes(int B, int Hq, int Hkv, int Sq, int Sk, int D,
  * first call on a device and kept), so that one chunk's kernels overlap the next
  * chunk's copies in and the previous chunk's copies out; those streams start after
  * the work already enqueued on `stream` and `stream` continues after them, so the
- * call is ordered on `stream` like any other.  Host buffers must be pinned for the
+ * call is ordered on `stream` like any other (the library takes a lock while it enqueues,
+ * so calls from several host threads are safe; each call in flight needs its own staging).  Host buffers must be pinned for the
  * copies to be asynchronous and to overlap; the results are valid after the caller
  * synchronises `stream`.  Results are the same bits as vt_attn_fwd on the whole
  * problem whenever the chunks get the same kernel (see vt_attn_fwd_kernel_kind).
@@ -400,12 +409,24 @@ int vt_attn_fwd_bwd_host_f16(const void *q_host, const void *k_host, const void 
 /*
  * Every wait inside the kernels is bounded.  If one expires, the kernel records
  * where in a per-device status word, lets all its warps leave, and returns
- * normally; outputs of that launch are then undefined.  This call synchronises
- * `stream`, reads the word of the current device, clears it, and returns
- * VT_ATTN_OK or VT_ATTN_ERR_DEVICE_TIMEOUT.  detail (host, may be NULL) receives
- * the raw word: bits 0-7 kernel id, 8-15 waiting role, 16-31 tile index.
+ * normally; outputs of that launch are then undefined.  The word is sticky: the
+ * first expired wait stays recorded until it is cleared.
+ *
+ * vt_attn_device_status is the convenient, BLOCKING form (the one entry point of this
+ * library that synchronises): it waits for `stream`, reads the word of the current
+ * device, clears it if set (waiting once more), and returns VT_ATTN_OK or
+ * VT_ATTN_ERR_DEVICE_TIMEOUT.  detail (host, may be NULL) receives the raw word: bits
+ * 0-7 kernel id, 8-15 waiting role, 16-31 tile index.  Not for use during stream capture.
+ *
+ * vt_attn_device_status_async and vt_attn_device_status_clear are the non-blocking
+ * pieces for callers that own their synchronisation points: the first enqueues a copy
+ * of the word into *word_host (host memory, pinned for the copy to be asynchronous;
+ * valid once the caller has synchronised `stream`; 0 = no wait expired), the second
+ * enqueues the reset of the word.  Neither synchronises.
  */
 int vt_attn_device_status(unsigned int *detail, void *stream);
+int vt_attn_device_status_async(unsigned int *word_host, void *stream);
+int vt_attn_device_status_clear(void *stream);
 
 /*
  * Static facts about the build, written to info[0..n) (host): [0] ABI version,

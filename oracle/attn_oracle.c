@@ -99,6 +99,19 @@ int attn_oracle_num_threads(void)
 #endif
 }
 
+/* Sets the number of OpenMP threads later calls use (n >= 1); returns the value now in force.  Threading only decides
+ * which core computes which (b, g) slice, never the arithmetic inside one: a test checks the results are the same bits. */
+int attn_oracle_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    if (n >= 1) omp_set_num_threads(n);
+    return omp_get_max_threads();
+#else
+    (void)n;
+    return 1;
+#endif
+}
+
 static int bad_shape(int B, int Hq, int Hkv, int Sq, int Sk, int D)
 {
     return B <= 0 || Hq <= 0 || Hkv <= 0 || Sq <= 0 || Sk <= 0 || D <= 0 || (Hq % Hkv) != 0;

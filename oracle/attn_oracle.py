@@ -46,6 +46,8 @@ def _load():
         lib = ctypes.CDLL(build())
         dims = [ctypes.c_int] * 6
         lib.attn_oracle_num_threads.restype = ctypes.c_int
+        lib.attn_oracle_set_num_threads.restype = ctypes.c_int
+        lib.attn_oracle_set_num_threads.argtypes = [ctypes.c_int]
         lib.attn_oracle_fwd.restype = ctypes.c_int
         lib.attn_oracle_fwd.argtypes = [_DP] * 5 + dims + [ctypes.c_int, ctypes.c_double]
         lib.attn_oracle_probs.restype = ctypes.c_int
@@ -60,6 +62,11 @@ def _load():
 def num_threads() -> int:
     """Threads the oracle's OpenMP loops will use."""
     return int(_load().attn_oracle_num_threads())
+
+
+def set_num_threads(n: int) -> int:
+    """Use ``n`` OpenMP threads from now on; returns the number in force."""
+    return int(_load().attn_oracle_set_num_threads(int(n)))
 
 
 def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:

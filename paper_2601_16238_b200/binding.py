@@ -62,6 +62,8 @@ EXPORTS = {
     "vt_attn_fwd_host_f16": (_i, [_vp] * 5 + _DIMS + [_i, _f, _vp, _sz, _vp]),
     "vt_attn_fwd_bwd_host_f16": (_i, [_vp] * 9 + _DIMS + [_i, _f, _vp, _sz, _vp]),
     "vt_attn_device_status": (_i, [ctypes.POINTER(ctypes.c_uint), _vp]),
+    "vt_attn_device_status_async": (_i, [_vp, _vp]),
+    "vt_attn_device_status_clear": (_i, [_vp]),
     "vt_attn_get_info": (_i, [ctypes.POINTER(_i), _i]),
     "vt_attn_selftest_tile": (_i, [_vp] * 5 + [_i, _f, _vp]),
     "vt_attn_selftest_timeout": (_i, [ctypes.c_uint, _vp]),
@@ -103,26 +105,58 @@ def _check(rc: int, what: str):
         raise VtAttnError(rc, f"{what}: {msg}" + (f" ({detail})" if detail else ""))
 
 
-def _stream(stream):
+def _stream(stream, device=None):
     import torch
     if stream is None:
-        stream = torch.cuda.current_stream()
+        stream = torch.cuda.current_stream(device)
     return stream.cuda_stream         # a plain int: ctypes converts it through the declared c_void_p argtype
 
 
-def _dims(q, k):
-    B, Hq, Sq, D = q.shape
-    _, Hkv, Sk, _ = k.shape
-    return int(B), int(Hq), int(Hkv), int(Sq), int(Sk), int(D)
+def _call(device, fn, *args):
+    """Run the C entry point with `device` current: the library launches on the current device."""
+    import torch
+    if device.type == "cuda" and device.index is not None and device.index != torch.cuda.current_device():
+        with torch.cuda.device(device):
+            return fn(*args)
+    return fn(*args)
 
 
 def _p(t):
     return t.data_ptr()               # plain int, converted by the declared argtypes (cheaper than a c_void_p object)
 
 
-def _require(t, dtype, name, device_type="cuda"):
+def _require(t, dtype, name, device_type="cuda", shape=None, device=None):
+    """Raise ValueError unless `t` is a contiguous tensor of `dtype` on a `device_type` device (the very `device`, if
+    given) with exactly `shape` (if given).  Every tensor is checked BEFORE the library is entered: the kernels trust the
+    sizes they are told, and a short tensor would be read or written past its end on the GPU."""
+    if shape is not None and tuple(t.shape) != tuple(shape):
+        raise ValueError(f"{name}: expected shape {tuple(shape)}, got {tuple(t.shape)}")
     if t.dtype != dtype or not t.is_contiguous() or t.device.type != device_type:
         raise ValueError(f"{name}: expected a contiguous {dtype} tensor on {device_type}")
+    if device is not None and t.device != device:
+        raise ValueError(f"{name}: on {t.device}, the other tensors are on {device}")
+
+
+def _dims(q, k, v=None, own_dv=False):
+    """(B, Hq, Hkv, Sq, Sk, D) after checking that q, k (and v) are 4-d tensors whose shapes agree with one another."""
+    if q.dim() != 4 or k.dim() != 4:
+        raise ValueError("q and k must be [B, H, S, D]")
+    B, Hq, Sq, D = (int(x) for x in q.shape)
+    Bk, Hkv, Sk, Dk = (int(x) for x in k.shape)
+    if Bk != B or Dk != D:
+        raise ValueError(f"q {tuple(q.shape)} and k {tuple(k.shape)} disagree on the batch or the head dimension")
+    if Hkv <= 0 or Hq % Hkv != 0:
+        raise ValueError(f"Hq = {Hq} is not a multiple of Hkv = {Hkv}")
+    if v is not None and (v.dim() != 4 or tuple(v.shape[:3]) != (B, Hkv, Sk) or (not own_dv and int(v.shape[3]) != D)):
+        raise ValueError(f"v {tuple(v.shape)} does not match k {tuple(k.shape)}")
+    return B, Hq, Hkv, Sq, Sk, D
+
+
+def _inputs(dtype, device_type, q, **others):
+    """dtype / contiguity / device of the input tensors (their shapes were checked by _dims)."""
+    _require(q, dtype, "q", device_type)
+    for name, t in others.items():
+        _require(t, dtype, name, device_type, device=q.device)
 
 
 def _mask_mode(causal) -> int:
@@ -133,17 +167,26 @@ def _mask_mode(causal) -> int:
     return mode
 
 
-def _fwd(entry: str, dtype, q, k, v, causal, scale, o, lse, stream):
+def _outputs_fwd(q, o, lse, o_shape, lse_shape):
     import torch
-    lib = load_library()
-    for t, n in ((q, "q"), (k, "k"), (v, "v")):
-        _require(t, dtype, n)
-    dims = _dims(q, k)
     if o is None:
-        o = torch.empty_like(q)
+        o = torch.empty(o_shape, dtype=q.dtype, device=q.device)
+    else:
+        _require(o, q.dtype, "o", shape=o_shape, device=q.device)
     if lse is None:
-        lse = torch.empty(q.shape[:3], dtype=torch.float32, device=q.device)
-    rc = getattr(lib, entry)(_p(q), _p(k), _p(v), _p(o), _p(lse), *dims, _mask_mode(causal), float(scale), _stream(stream))
+        lse = torch.empty(lse_shape, dtype=torch.float32, device=q.device)
+    else:
+        _require(lse, torch.float32, "lse", shape=lse_shape, device=q.device)
+    return o, lse
+
+
+def _fwd(entry: str, dtype, q, k, v, causal, scale, o, lse, stream):
+    lib = load_library()
+    dims = _dims(q, k, v)
+    o, lse = _outputs_fwd(q, o, lse, q.shape, q.shape[:3])
+    _inputs(dtype, "cuda", q, k=k, v=v)
+    rc = _call(q.device, getattr(lib, entry), _p(q), _p(k), _p(v), _p(o), _p(lse), *dims, _mask_mode(causal), float(scale),
+               _stream(stream, q.device))
     _check(rc, entry)
     return o, lse
 
@@ -155,17 +198,13 @@ def vt_attn_fwd(q, k, v, causal: bool, scale: float, o=None, lse=None, stream=No
 
 
 def _fwd_dv(name, dtype, q, k, v, causal, scale, o, lse, stream):
-    import torch
     lib = load_library()
-    for t, n in ((q, "q"), (k, "k"), (v, "v")):
-        _require(t, dtype, n)
-    dims = _dims(q, k)
+    dims = _dims(q, k, v, own_dv=True)
     Dv = int(v.shape[-1])
-    if o is None:
-        o = torch.empty(q.shape[:3] + (Dv,), dtype=q.dtype, device=q.device)
-    if lse is None:
-        lse = torch.empty(q.shape[:3], dtype=torch.float32, device=q.device)
-    rc = getattr(lib, name)(_p(q), _p(k), _p(v), _p(o), _p(lse), *dims, Dv, _mask_mode(causal), float(scale), _stream(stream))
+    o, lse = _outputs_fwd(q, o, lse, tuple(q.shape[:3]) + (Dv,), q.shape[:3])
+    _inputs(dtype, "cuda", q, k=k, v=v)
+    rc = _call(q.device, getattr(lib, name), _p(q), _p(k), _p(v), _p(o), _p(lse), *dims, Dv, _mask_mode(causal), float(scale),
+               _stream(stream, q.device))
     _check(rc, name)
     return o, lse
 
@@ -211,21 +250,23 @@ def vt_attn_fwd_splitkv_plan(B, Hq, Hkv, Sq, Sk, D, n_splits=0):
     return used.value, bool(share.value)
 
 
-def _splitkv(entry: str, dtype, q, k, v, causal, scale, n_splits, o, lse, workspace, stream):
+def _workspace(workspace, need, device):
     import torch
-    lib = load_library()
-    for t, n in ((q, "q"), (k, "k"), (v, "v")):
-        _require(t, dtype, n)
-    dims = _dims(q, k)
-    if o is None:
-        o = torch.empty_like(q)
-    if lse is None:
-        lse = torch.empty(q.shape[:3], dtype=torch.float32, device=q.device)
     if workspace is None:
-        need = lib.vt_attn_fwd_splitkv_workspace_bytes(*dims, int(n_splits))
-        workspace = torch.empty(max(256, need), dtype=torch.uint8, device=q.device)
-    rc = getattr(lib, entry)(_p(q), _p(k), _p(v), _p(o), _p(lse), *dims, _mask_mode(causal), float(scale), int(n_splits),
-                             _p(workspace), workspace.numel() * workspace.element_size(), _stream(stream))
+        return torch.empty(max(256, int(need)), dtype=torch.uint8, device=device)
+    if not workspace.is_contiguous() or workspace.device != device:
+        raise ValueError(f"workspace: expected a contiguous tensor on {device}")
+    return workspace
+
+
+def _splitkv(entry: str, dtype, q, k, v, causal, scale, n_splits, o, lse, workspace, stream):
+    lib = load_library()
+    dims = _dims(q, k, v)
+    o, lse = _outputs_fwd(q, o, lse, q.shape, q.shape[:3])
+    _inputs(dtype, "cuda", q, k=k, v=v)
+    workspace = _workspace(workspace, 0 if workspace is not None else lib.vt_attn_fwd_splitkv_workspace_bytes(*dims, int(n_splits)), q.device)
+    rc = _call(q.device, getattr(lib, entry), _p(q), _p(k), _p(v), _p(o), _p(lse), *dims, _mask_mode(causal), float(scale),
+               int(n_splits), _p(workspace), workspace.numel() * workspace.element_size(), _stream(stream, q.device))
     _check(rc, entry)
     return o, lse
 
@@ -242,21 +283,34 @@ def vt_attn_fwd_splitkv_f16(q, k, v, causal, scale: float, n_splits: int = 0, o=
     return _splitkv("vt_attn_fwd_splitkv_f16", torch.float16, q, k, v, causal, scale, n_splits, o, lse, workspace, stream)
 
 
+def _shapes(*items):
+    """(tensor or None, name, shape) triples: every tensor given has exactly that shape."""
+    for t, name, shape in items:
+        if t is not None and tuple(t.shape) != tuple(shape):
+            raise ValueError(f"{name}: expected shape {tuple(shape)}, got {tuple(t.shape)}")
+
+
+def _grad_out(t, like, name):
+    import torch
+    if t is None:
+        return torch.empty_like(like)
+    _require(t, like.dtype, name, shape=like.shape, device=like.device)
+    return t
+
+
 def _bwd(entry: str, dtype, q, k, v, o, d_o, lse, causal, scale, dq, dk, dv, workspace, stream):
     import torch
     lib = load_library()
-    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (d_o, "d_o")):
-        _require(t, dtype, n)
-    _require(lse, torch.float32, "lse")
-    dims = _dims(q, k)
-    dq = torch.empty_like(q) if dq is None else dq
-    dk = torch.empty_like(k) if dk is None else dk
-    dv = torch.empty_like(v) if dv is None else dv
-    if workspace is None:
-        workspace = torch.empty(max(256, lib.vt_attn_bwd_workspace_bytes(*dims)), dtype=torch.uint8, device=q.device)
-    rc = getattr(lib, entry)(_p(q), _p(k), _p(v), _p(o), _p(d_o), _p(lse), _p(dq), _p(dk), _p(dv), *dims,
-                             _mask_mode(causal), float(scale), _p(workspace), workspace.numel() * workspace.element_size(),
-                             _stream(stream))
+    dims = _dims(q, k, v)
+    _shapes((o, "o", q.shape), (d_o, "d_o", q.shape), (lse, "lse", q.shape[:3]), (dq, "dq", q.shape), (dk, "dk", k.shape),
+            (dv, "dv", v.shape))
+    _inputs(dtype, "cuda", q, k=k, v=v, o=o, d_o=d_o)
+    _require(lse, torch.float32, "lse", device=q.device)
+    dq, dk, dv = _grad_out(dq, q, "dq"), _grad_out(dk, k, "dk"), _grad_out(dv, v, "dv")
+    workspace = _workspace(workspace, 0 if workspace is not None else lib.vt_attn_bwd_workspace_bytes(*dims), q.device)
+    rc = _call(q.device, getattr(lib, entry), _p(q), _p(k), _p(v), _p(o), _p(d_o), _p(lse), _p(dq), _p(dk), _p(dv), *dims,
+               _mask_mode(causal), float(scale), _p(workspace), workspace.numel() * workspace.element_size(),
+               _stream(stream, q.device))
     _check(rc, entry)
     return dq, dk, dv
 
@@ -276,12 +330,15 @@ def vt_attn_bwd_f16(q, k, v, o, d_o, lse, causal: bool, scale: float, dq=None, d
 
 
 def _bwd_static(name, dtype, q, k, v, o, d_o, lse, causal, scale, dq, dk, dv, stream):
+    import torch
     lib = load_library()
-    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (d_o, "d_o"), (dq, "dq"), (dk, "dk"), (dv, "dv")):
-        _require(t, dtype, n)
-    dims = _dims(q, k)
-    rc = getattr(lib, name)(_p(q), _p(k), _p(v), _p(o), _p(d_o), _p(lse), _p(dq), _p(dk), _p(dv), *dims,
-                            _mask_mode(causal), float(scale), _stream(stream))
+    dims = _dims(q, k, v)
+    _shapes((o, "o", q.shape), (d_o, "d_o", q.shape), (lse, "lse", q.shape[:3]), (dq, "dq", q.shape), (dk, "dk", k.shape),
+            (dv, "dv", v.shape))
+    _inputs(dtype, "cuda", q, k=k, v=v, o=o, d_o=d_o, dq=dq, dk=dk, dv=dv)
+    _require(lse, torch.float32, "lse", device=q.device)
+    rc = _call(q.device, getattr(lib, name), _p(q), _p(k), _p(v), _p(o), _p(d_o), _p(lse), _p(dq), _p(dk), _p(dv), *dims,
+               _mask_mode(causal), float(scale), _stream(stream, q.device))
     _check(rc, name)
     return dq, dk, dv
 
@@ -300,26 +357,34 @@ def vt_attn_bwd_static_scratch_f16(q, k, v, o, d_o, lse, causal: bool, scale: fl
     return _bwd_static("vt_attn_bwd_static_scratch_f16", torch.float16, q, k, v, o, d_o, lse, causal, scale, dq, dk, dv, stream)
 
 
-def _varlen_dims(q, k, cu_q, max_sq, max_sk):
-    total_q, Hq, D = q.shape
-    total_k, Hkv, _ = k.shape
-    return int(cu_q.numel()) - 1, int(Hq), int(Hkv), int(total_q), int(total_k), int(max_sq), int(max_sk), int(D)
+def _varlen_dims(q, k, v, cu_q, cu_k, max_sq, max_sk, dtype, **more):
+    """(n_seqs, Hq, Hkv, total_q, total_k, max_sq, max_sk, D) after checking the packed tensors against one another.
+    `more`: name -> (tensor or None, shape) of further tensors whose shapes are checked before any dtype / device."""
+    import torch
+    if q.dim() != 3 or k.dim() != 3:
+        raise ValueError("packed q and k must be [total, H, D]")
+    total_q, Hq, D = (int(x) for x in q.shape)
+    total_k, Hkv, Dk = (int(x) for x in k.shape)
+    if Dk != D:
+        raise ValueError("q and k disagree on the head dimension")
+    if Hkv <= 0 or Hq % Hkv != 0:
+        raise ValueError(f"Hq = {Hq} is not a multiple of Hkv = {Hkv}")
+    if cu_q.dim() != 1 or cu_q.numel() < 1 or cu_k.shape != cu_q.shape:
+        raise ValueError("cu_seqlens_q and cu_seqlens_k must be 1-d with n_seqs + 1 entries each")
+    _shapes((v, "v", k.shape), *((t, n, shp) for n, (t, shp) in more.items()))
+    _inputs(dtype, "cuda", q, k=k, v=v)
+    _require(cu_q, torch.int32, "cu_seqlens_q", device=q.device)
+    _require(cu_k, torch.int32, "cu_seqlens_k", device=q.device)
+    return int(cu_q.numel()) - 1, Hq, Hkv, total_q, total_k, int(max_sq), int(max_sk), D
 
 
 def _fwd_varlen(entry: str, dtype, q, k, v, cu_seqlens_q, cu_seqlens_k, max_sq, max_sk, causal, scale, o, lse, stream):
-    import torch
     lib = load_library()
-    for t, n in ((q, "q"), (k, "k"), (v, "v")):
-        _require(t, dtype, n)
-    _require(cu_seqlens_q, torch.int32, "cu_seqlens_q")
-    _require(cu_seqlens_k, torch.int32, "cu_seqlens_k")
-    dims = _varlen_dims(q, k, cu_seqlens_q, max_sq, max_sk)
-    if o is None:
-        o = torch.empty_like(q)
-    if lse is None:
-        lse = torch.empty((q.shape[1], q.shape[0]), dtype=torch.float32, device=q.device)
-    rc = getattr(lib, entry)(_p(q), _p(k), _p(v), _p(o), _p(lse), _p(cu_seqlens_q), _p(cu_seqlens_k), *dims,
-                             _mask_mode(causal), float(scale), _stream(stream))
+    dims = _varlen_dims(q, k, v, cu_seqlens_q, cu_seqlens_k, max_sq, max_sk, dtype,
+                        o=(o, q.shape), lse=(lse, (q.shape[1], q.shape[0])))
+    o, lse = _outputs_fwd(q, o, lse, q.shape, (q.shape[1], q.shape[0]))
+    rc = _call(q.device, getattr(lib, entry), _p(q), _p(k), _p(v), _p(o), _p(lse), _p(cu_seqlens_q), _p(cu_seqlens_k), *dims,
+               _mask_mode(causal), float(scale), _stream(stream, q.device))
     _check(rc, entry)
     return o, lse
 
@@ -349,23 +414,15 @@ def vt_attn_fwd_splitkv_varlen_plan(n_seqs, Hq, Hkv, total_k, max_sq, max_sk, D,
 
 
 def _splitkv_varlen(name, dtype, q, k, v, cu_seqlens_q, cu_seqlens_k, max_sq, max_sk, causal, scale, n_splits, o, lse, workspace, stream):
-    import torch
     lib = load_library()
-    for t, n in ((q, "q"), (k, "k"), (v, "v")):
-        _require(t, dtype, n)
-    _require(cu_seqlens_q, torch.int32, "cu_seqlens_q")
-    _require(cu_seqlens_k, torch.int32, "cu_seqlens_k")
-    dims = _varlen_dims(q, k, cu_seqlens_q, max_sq, max_sk)       # n_seqs, Hq, Hkv, total_q, total_k, max_sq, max_sk, D
-    if o is None:
-        o = torch.empty_like(q)
-    if lse is None:
-        lse = torch.empty((q.shape[1], q.shape[0]), dtype=torch.float32, device=q.device)
-    if workspace is None:
-        need = lib.vt_attn_fwd_splitkv_varlen_workspace_bytes(dims[0], dims[1], dims[2], dims[3], dims[5], dims[6], dims[7], int(n_splits))
-        workspace = torch.empty(max(256, need), dtype=torch.uint8, device=q.device)
-    rc = getattr(lib, name)(_p(q), _p(k), _p(v), _p(o), _p(lse), _p(cu_seqlens_q), _p(cu_seqlens_k), *dims,
-                            _mask_mode(causal), float(scale), int(n_splits), _p(workspace),
-                            workspace.numel() * workspace.element_size(), _stream(stream))
+    dims = _varlen_dims(q, k, v, cu_seqlens_q, cu_seqlens_k, max_sq, max_sk, dtype,      # n_seqs, Hq, Hkv, total_q, total_k, max_sq, max_sk, D
+                        o=(o, q.shape), lse=(lse, (q.shape[1], q.shape[0])))
+    o, lse = _outputs_fwd(q, o, lse, q.shape, (q.shape[1], q.shape[0]))
+    need = 0 if workspace is not None else lib.vt_attn_fwd_splitkv_varlen_workspace_bytes(dims[0], dims[1], dims[2], dims[3], dims[5], dims[6], dims[7], int(n_splits))
+    workspace = _workspace(workspace, need, q.device)
+    rc = _call(q.device, getattr(lib, name), _p(q), _p(k), _p(v), _p(o), _p(lse), _p(cu_seqlens_q), _p(cu_seqlens_k), *dims,
+               _mask_mode(causal), float(scale), int(n_splits), _p(workspace),
+               workspace.numel() * workspace.element_size(), _stream(stream, q.device))
     _check(rc, name)
     return o, lse
 
@@ -389,23 +446,27 @@ def vt_attn_fwd_splitkv_varlen_f16(q, k, v, cu_seqlens_q, cu_seqlens_k, max_sq: 
 def vt_attn_merge_partial(o_acc, lse_acc, o_part, lse_part, first: bool, stream=None):
     """Fold one partial forward result (bf16 O, fp32 LSE over one block of keys) into the fp32 running result."""
     import torch
-    _require(o_acc, torch.float32, "o_acc")
-    _require(lse_acc, torch.float32, "lse_acc")
+    if o_part.dim() < 2:
+        raise ValueError("o_part must be [..., rows, D]")
+    _shapes((o_acc, "o_acc", o_part.shape), (lse_part, "lse_part", o_part.shape[:-1]), (lse_acc, "lse_acc", o_part.shape[:-1]))
     _require(o_part, torch.bfloat16, "o_part")
-    _require(lse_part, torch.float32, "lse_part")
+    _require(o_acc, torch.float32, "o_acc", shape=o_part.shape, device=o_part.device)
+    _require(lse_part, torch.float32, "lse_part", shape=o_part.shape[:-1], device=o_part.device)
+    _require(lse_acc, torch.float32, "lse_acc", shape=o_part.shape[:-1], device=o_part.device)
     D = int(o_part.shape[-1])
-    rc = load_library().vt_attn_merge_partial(_p(o_acc), _p(lse_acc), _p(o_part), _p(lse_part), o_part.numel() // D, D,
-                                              int(bool(first)), _stream(stream))
+    rc = _call(o_part.device, load_library().vt_attn_merge_partial, _p(o_acc), _p(lse_acc), _p(o_part), _p(lse_part),
+               o_part.numel() // D, D, int(bool(first)), _stream(stream, o_part.device))
     _check(rc, "vt_attn_merge_partial")
 
 
 def vt_attn_accumulate_partial(acc, part, first: bool, stream=None):
     """acc (fp32) += part (bf16); acc = part when ``first``."""
     import torch
-    _require(acc, torch.float32, "acc")
     _require(part, torch.bfloat16, "part")
+    _require(acc, torch.float32, "acc", shape=part.shape, device=part.device)
     D = int(part.shape[-1])
-    rc = load_library().vt_attn_accumulate_partial(_p(acc), _p(part), part.numel() // D, D, int(bool(first)), _stream(stream))
+    rc = _call(part.device, load_library().vt_attn_accumulate_partial, _p(acc), _p(part), part.numel() // D, D,
+               int(bool(first)), _stream(stream, part.device))
     _check(rc, "vt_attn_accumulate_partial")
 
 
@@ -415,8 +476,11 @@ def vt_attn_merge_finish(o_acc, o=None, stream=None):
     _require(o_acc, torch.float32, "o_acc")
     if o is None:
         o = torch.empty(o_acc.shape, dtype=torch.bfloat16, device=o_acc.device)
+    else:
+        _require(o, torch.bfloat16, "o", shape=o_acc.shape, device=o_acc.device)
     D = int(o_acc.shape[-1])
-    rc = load_library().vt_attn_merge_finish(_p(o_acc), _p(o), o_acc.numel() // D, D, _stream(stream))
+    rc = _call(o_acc.device, load_library().vt_attn_merge_finish, _p(o_acc), _p(o), o_acc.numel() // D, D,
+               _stream(stream, o_acc.device))
     _check(rc, "vt_attn_merge_finish")
     return o
 
@@ -429,19 +493,17 @@ def _bwd_varlen(entry: str, dtype, q, k, v, o, d_o, lse, cu_seqlens_q, cu_seqlen
                 workspace, stream):
     import torch
     lib = load_library()
-    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o"), (d_o, "d_o")):
-        _require(t, dtype, n)
-    _require(lse, torch.float32, "lse")
-    dims = _varlen_dims(q, k, cu_seqlens_q, max_sq, max_sk)
-    dq = torch.empty_like(q) if dq is None else dq
-    dk = torch.empty_like(k) if dk is None else dk
-    dv = torch.empty_like(v) if dv is None else dv
-    if workspace is None:
-        workspace = torch.empty(max(256, lib.vt_attn_bwd_varlen_workspace_bytes(dims[1], dims[3])), dtype=torch.uint8,
-                                device=q.device)
-    rc = getattr(lib, entry)(_p(q), _p(k), _p(v), _p(o), _p(d_o), _p(lse), _p(dq), _p(dk), _p(dv), _p(cu_seqlens_q),
-                             _p(cu_seqlens_k), *dims, _mask_mode(causal), float(scale), _p(workspace),
-                             workspace.numel() * workspace.element_size(), _stream(stream))
+    lse_shape = (q.shape[1], q.shape[0]) if q.dim() == 3 else None
+    dims = _varlen_dims(q, k, v, cu_seqlens_q, cu_seqlens_k, max_sq, max_sk, dtype, o=(o, q.shape), d_o=(d_o, q.shape),
+                        lse=(lse, lse_shape), dq=(dq, q.shape), dk=(dk, k.shape), dv=(dv, k.shape))
+    _require(o, dtype, "o", shape=q.shape, device=q.device)
+    _require(d_o, dtype, "d_o", shape=q.shape, device=q.device)
+    _require(lse, torch.float32, "lse", shape=(q.shape[1], q.shape[0]), device=q.device)
+    dq, dk, dv = _grad_out(dq, q, "dq"), _grad_out(dk, k, "dk"), _grad_out(dv, v, "dv")
+    workspace = _workspace(workspace, 0 if workspace is not None else lib.vt_attn_bwd_varlen_workspace_bytes(dims[1], dims[3]), q.device)
+    rc = _call(q.device, getattr(lib, entry), _p(q), _p(k), _p(v), _p(o), _p(d_o), _p(lse), _p(dq), _p(dk), _p(dv),
+               _p(cu_seqlens_q), _p(cu_seqlens_k), *dims, _mask_mode(causal), float(scale), _p(workspace),
+               workspace.numel() * workspace.element_size(), _stream(stream, q.device))
     _check(rc, entry)
     return dq, dk, dv
 
@@ -467,24 +529,29 @@ def vt_attn_host_staging_bytes(B, Hq, Hkv, Sq, Sk, D, with_backward: bool) -> in
 
 
 def _fwd_host(name, dtype, q, k, v, o, lse, causal, scale, staging, stream):
+    import torch
     lib = load_library()
-    for t, n in ((q, "q"), (k, "k"), (v, "v"), (o, "o")):
-        if t.dtype != dtype or t.is_cuda or not t.is_contiguous():
-            raise ValueError(f"{n} must be a contiguous {dtype} host tensor")
-    dims = _dims(q, k)
-    rc = getattr(lib, name)(_p(q), _p(k), _p(v), _p(o), _p(lse), *dims, _mask_mode(causal), float(scale),
-                            _p(staging), staging.numel(), _stream(stream))
+    dims = _dims(q, k, v)
+    _shapes((o, "o", q.shape), (lse, "lse", q.shape[:3]))
+    _inputs(dtype, "cpu", q, k=k, v=v, o=o)
+    _require(lse, torch.float32, "lse", "cpu")
+    _require(staging, torch.uint8, "staging")
+    rc = _call(staging.device, getattr(lib, name), _p(q), _p(k), _p(v), _p(o), _p(lse), *dims, _mask_mode(causal), float(scale),
+               _p(staging), staging.numel(), _stream(stream, staging.device))
     _check(rc, name)
 
 
 def _fwd_bwd_host(name, dtype, q, k, v, d_o, o, lse, dq, dk, dv, causal, scale, staging, stream):
+    import torch
     lib = load_library()
-    for t, n in ((q, "q"), (k, "k"), (v, "v"), (d_o, "d_o"), (o, "o"), (dq, "dq"), (dk, "dk"), (dv, "dv")):
-        if t.dtype != dtype or t.is_cuda or not t.is_contiguous():
-            raise ValueError(f"{n} must be a contiguous {dtype} host tensor")
-    dims = _dims(q, k)
-    rc = getattr(lib, name)(_p(q), _p(k), _p(v), _p(d_o), _p(o), _p(lse), _p(dq), _p(dk), _p(dv), *dims,
-                            _mask_mode(causal), float(scale), _p(staging), staging.numel(), _stream(stream))
+    dims = _dims(q, k, v)
+    _shapes((d_o, "d_o", q.shape), (o, "o", q.shape), (dq, "dq", q.shape), (dk, "dk", k.shape), (dv, "dv", v.shape),
+            (lse, "lse", q.shape[:3]))
+    _inputs(dtype, "cpu", q, k=k, v=v, d_o=d_o, o=o, dq=dq, dk=dk, dv=dv)
+    _require(lse, torch.float32, "lse", "cpu")
+    _require(staging, torch.uint8, "staging")
+    rc = _call(staging.device, getattr(lib, name), _p(q), _p(k), _p(v), _p(d_o), _p(o), _p(lse), _p(dq), _p(dk), _p(dv), *dims,
+               _mask_mode(causal), float(scale), _p(staging), staging.numel(), _stream(stream, staging.device))
     _check(rc, name)
 
 
@@ -518,6 +585,20 @@ def vt_attn_device_status(stream=None):
     detail = ctypes.c_uint(0)
     rc = lib.vt_attn_device_status(ctypes.byref(detail), _stream(stream))
     return int(rc), int(detail.value)
+
+
+def vt_attn_device_status_async(word_host, stream=None):
+    """Enqueue a copy of the status word into ``word_host`` (a pinned int32 host tensor of one element).  No
+    synchronisation: the value is valid after the caller has synchronised the stream (0: no wait expired)."""
+    import torch
+    if word_host.is_cuda or word_host.dtype != torch.int32 or word_host.numel() != 1:
+        raise ValueError("word_host: expected a one-element int32 host tensor")
+    _check(load_library().vt_attn_device_status_async(_p(word_host), _stream(stream)), "vt_attn_device_status_async")
+
+
+def vt_attn_device_status_clear(stream=None):
+    """Enqueue the reset of the status word.  No synchronisation."""
+    _check(load_library().vt_attn_device_status_clear(_stream(stream)), "vt_attn_device_status_clear")
 
 
 def vt_attn_get_info():

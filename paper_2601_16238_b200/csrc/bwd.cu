@@ -834,13 +834,13 @@ static int launch_bwd(const BwdMaps &m, BwdParams prm, const __nv_bfloat16 *o, c
                       cudaStream_t stream)
 {
     int rc;
-    static bool configured[64] = {};
+    static std::atomic<bool> configured[64];     // set-up is idempotent: two threads may both do it, neither may read a torn flag
     int dev = 0;
     cudaGetDevice(&dev);
-    if (!configured[dev & 63]) {
+    if (!configured[dev & 63].load(std::memory_order_acquire)) {
         if ((rc = set_smem(bwd_dkdv_kernel<D, CAUSAL, PACKED, F16>, DkdvSmem<D>::BYTES, "cudaFuncSetAttribute(dkdv)")) != VT_ATTN_OK) return rc;
         if ((rc = set_smem(bwd_dq_kernel<D, CAUSAL, PACKED, F16>, DqSmem<D>::BYTES, "cudaFuncSetAttribute(dq)")) != VT_ATTN_OK) return rc;
-        configured[dev & 63] = true;
+        configured[dev & 63].store(true, std::memory_order_release);
     }
 
     const long long n_rows = PACKED ? static_cast<long long>(prm.total_q) * prm.Hq : static_cast<long long>(B) * prm.Hq * prm.Sq;

@@ -235,4 +235,23 @@ int vt_attn_device_status(unsigned int *detail, void *stream)
     return VT_ATTN_OK;
 }
 
+int vt_attn_device_status_async(unsigned int *word_host, void *stream)
+{
+    if (!word_host) return VT_ATTN_ERR_INVALID_ARGUMENT;
+    unsigned int *p = vt::status_word_ptr();
+    if (!p) return VT_ATTN_ERR_CUDA;
+    cudaError_t e = cudaMemcpyAsync(word_host, p, sizeof(unsigned int), cudaMemcpyDeviceToHost, static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return vt::cuda_fail(e, "cudaMemcpyAsync(status)");
+    return VT_ATTN_OK;
+}
+
+int vt_attn_device_status_clear(void *stream)
+{
+    unsigned int *p = vt::status_word_ptr();
+    if (!p) return VT_ATTN_ERR_CUDA;
+    cudaError_t e = cudaMemsetAsync(p, 0, sizeof(unsigned int), static_cast<cudaStream_t>(stream));
+    if (e != cudaSuccess) return vt::cuda_fail(e, "cudaMemsetAsync(status)");
+    return VT_ATTN_OK;
+}
+
 }  // extern "C"

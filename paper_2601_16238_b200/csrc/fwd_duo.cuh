@@ -350,13 +350,13 @@ template <int D, bool F16>
 static int launch_fwd_duo(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const FwdParams &prm,
                           int n_blocks, cudaStream_t stream)
 {
-    static bool configured[64] = {};
+    static std::atomic<bool> configured[64];     // set-up is idempotent: two threads may both do it, neither may read a torn flag
     int dev = 0;
     cudaGetDevice(&dev);
-    if (!configured[dev & 63]) {
+    if (!configured[dev & 63].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(attn_fwd_duo_kernel<D, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, DuoSmem<D>::BYTES);
         if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(fwd duo)");
-        configured[dev & 63] = true;
+        configured[dev & 63].store(true, std::memory_order_release);
     }
     attn_fwd_duo_kernel<D, F16><<<n_blocks, FWD_THREADS, DuoSmem<D>::BYTES, stream>>>(tq, tk, tv, prm);
     cudaError_t e = cudaGetLastError();

@@ -397,13 +397,13 @@ static int launch_fwd_pair(const CUtensorMap &tq, const CUtensorMap &tk, const C
                            int n_blocks, cudaStream_t stream)
 {
     using L = PairSmem<D>;
-    static bool configured[64] = {};
+    static std::atomic<bool> configured[64];     // set-up is idempotent: two threads may both do it, neither may read a torn flag
     int dev = 0;
     cudaGetDevice(&dev);
-    if (!configured[dev & 63]) {
+    if (!configured[dev & 63].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(attn_fwd_pair_kernel<D, CAUSAL, PACKED, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES);
         if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(fwd pair)");
-        configured[dev & 63] = true;
+        configured[dev & 63].store(true, std::memory_order_release);
     }
     attn_fwd_pair_kernel<D, CAUSAL, PACKED, F16><<<n_blocks, PAIR_THREADS, L::BYTES, stream>>>(tq, tk, tv, prm);
     cudaError_t e = cudaGetLastError();

@@ -129,6 +129,12 @@ template <int DD, bool F16>
 static int launch_split_packed(bool causal, bool hpack, const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const FwdParams &prm,
                                int nb, float *lse, int n_splits, int d, cudaStream_t st)
 {
+    // Query tokens of a sequence past max_sq are owned by no block and get no partial result.  Their partial LSEs are
+    // preset to all-ones bits (a NaN): fmaxf ignores a NaN operand, so the merge sees "no chunk saw a key" for exactly
+    // those rows and writes O = 0, LSE = -inf instead of reading uninitialised scratch.  Rows that are processed get a
+    // real partial LSE from every chunk's block (empty chunks write -inf), so the preset never mixes with real values.
+    cudaError_t e = cudaMemsetAsync(prm.lse_part, 0xFF, static_cast<size_t>(n_splits) * prm.n_rows * sizeof(float), st);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(partial LSE)");
     int rc;
     if (hpack) rc = causal ? launch_fwd<DD, true, true, true, true, F16>(tq, tk, tv, prm, nb, st) : launch_fwd<DD, false, true, true, true, F16>(tq, tk, tv, prm, nb, st);
     else rc = causal ? launch_fwd<DD, true, true, true, false, F16>(tq, tk, tv, prm, nb, st) : launch_fwd<DD, false, true, true, false, F16>(tq, tk, tv, prm, nb, st);

@@ -93,7 +93,8 @@ struct SideStreams {
     bool ready;
 };
 static SideStreams g_side[64];
-static std::mutex g_side_mutex;
+static std::mutex g_side_mutex;      // creation of the streams and events
+static std::mutex g_call_mutex;      // the fork / enqueue / join of one host-buffer call
 
 static int side_streams(SideStreams **out)
 {
@@ -134,6 +135,10 @@ static int run_chunked(bool f16, const HostArgs &h, int B, int Hq, int Hkv, int 
     SideStreams *ss = nullptr;
     int rc = side_streams(&ss);
     if (rc != VT_ATTN_OK) return rc;
+    // One call at a time per process forks onto and joins from the library's streams and events: a second thread's
+    // cudaEventRecord(start) between this thread's record and its waits would move this call's fork point.  Everything
+    // below only enqueues, so the lock is held for microseconds.
+    std::lock_guard<std::mutex> call_lock(g_call_mutex);
     cudaError_t e;
     if ((e = cudaEventRecord(ss->start, user)) != cudaSuccess) return cuda_fail(e, "cudaEventRecord");
     for (int i = 0; i < 2; ++i)

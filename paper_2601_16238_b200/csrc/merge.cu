@@ -9,26 +9,38 @@ namespace vt {
 
 // The kernels below give a thread 8 elements of a row (D / 8 threads per row, D a multiple of 8) and walk the
 // n_rows * D / 8 pieces with a grid-stride loop.
+//
+// merge_partial_kernel reads and rewrites lse_acc[row] in one launch, so every thread of a row must have read the old
+// value before one of them stores the new one.  The threads of a row are therefore padded to a power of two (`tpr_pad`,
+// at most 32): a row then never straddles a warp, the loop bounds are the same for all lanes of a warp, and a
+// __syncwarp() separates the row's loads from the store.  Lanes past the row's real D / 8 pieces only take part in the
+// barrier.
 __global__ void __launch_bounds__(256) merge_partial_kernel(float *__restrict__ o_acc, float *__restrict__ lse_acc,
                                                             const __nv_bfloat16 *__restrict__ o_part, const float *__restrict__ lse_part,
-                                                            long long n_rows, int D, int first)
+                                                            long long n_rows, int D, int tpr_pad, int first)
 {
     const int tpr = D / 8;
-    const long long n_pieces = n_rows * tpr;
-    for (long long i = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x; i < n_pieces; i += static_cast<long long>(gridDim.x) * 256) {
-        const long long row = i / tpr;
-        const int sub = static_cast<int>(i - row * tpr);
-        const float lp = lse_part[row];
-        const float la = first ? -INFINITY : lse_acc[row];
-        const float m = fmaxf(la, lp);
+    const long long n_slots = n_rows * tpr_pad;                         // a multiple of tpr_pad; rows are whole within a warp
+    const long long n_warp_slots = (n_slots + 31) / 32 * 32;            // warp-uniform loop bound
+    for (long long i = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x; i < n_warp_slots; i += static_cast<long long>(gridDim.x) * 256) {
+        const long long row = i / tpr_pad;
+        const int sub = static_cast<int>(i - row * tpr_pad);
+        const bool live = row < n_rows && sub < tpr;
         float wa = 0.0f, wp = 0.0f, ln = -INFINITY;
-        if (m != -INFINITY) {                        // at least one side saw a key
-            const float ea = __expf(la - m), ep = __expf(lp - m);      // exp(-inf) = 0
-            const float inv = 1.0f / (ea + ep);
-            wa = ea * inv;
-            wp = ep * inv;
-            ln = m + logf(ea + ep);
+        if (live) {
+            const float lp = lse_part[row];
+            const float la = first ? -INFINITY : lse_acc[row];
+            const float m = fmaxf(la, lp);
+            if (m != -INFINITY) {                        // at least one side saw a key
+                const float ea = __expf(la - m), ep = __expf(lp - m);      // exp(-inf) = 0
+                const float inv = 1.0f / (ea + ep);
+                wa = ea * inv;
+                wp = ep * inv;
+                ln = m + logf(ea + ep);
+            }
         }
+        __syncwarp();                                    // every lane of the row holds the old LSE before lane `sub == 0` replaces it
+        if (!live) continue;
         const uint4 pv = *reinterpret_cast<const uint4 *>(o_part + row * D + sub * 8);
         const uint32_t pw[4] = {pv.x, pv.y, pv.z, pv.w};
         float4 a0 = make_float4(0.f, 0.f, 0.f, 0.f), a1 = a0;
@@ -83,9 +95,16 @@ __global__ void __launch_bounds__(256) accumulate_kernel(float *__restrict__ acc
     }
 }
 
-static int merge_grid(long long n_rows, int D)
+static int pow2_at_least(int x)
 {
-    long long nb = (n_rows * (D / 8) + 255) / 256;
+    int p = 1;
+    while (p < x) p *= 2;
+    return p;
+}
+
+static int merge_grid(long long n_rows, int threads_per_row)
+{
+    long long nb = (n_rows * threads_per_row + 255) / 256;
     if (nb > NUM_SMS * 16) nb = NUM_SMS * 16;
     return static_cast<int>(nb);
 }
@@ -102,7 +121,8 @@ extern "C" int vt_attn_merge_partial(float *o_acc, float *lse_acc, const void *o
     if (rc != VT_ATTN_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const __nv_bfloat16 *part = static_cast<const __nv_bfloat16 *>(o_part);
-    merge_partial_kernel<<<merge_grid(n_rows, D), 256, 0, st>>>(o_acc, lse_acc, part, lse_part, n_rows, D, first);
+    const int tpr_pad = pow2_at_least(D / 8);
+    merge_partial_kernel<<<merge_grid(n_rows, tpr_pad), 256, 0, st>>>(o_acc, lse_acc, part, lse_part, n_rows, D, tpr_pad, first);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "merge_partial_kernel launch");
     return VT_ATTN_OK;
@@ -117,7 +137,7 @@ extern "C" int vt_attn_merge_finish(const float *o_acc, void *o, long long n_row
     if (rc != VT_ATTN_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     __nv_bfloat16 *out = static_cast<__nv_bfloat16 *>(o);
-    merge_finish_kernel<<<merge_grid(n_rows, D), 256, 0, st>>>(o_acc, out, n_rows, D);
+    merge_finish_kernel<<<merge_grid(n_rows, D / 8), 256, 0, st>>>(o_acc, out, n_rows, D);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "merge_finish_kernel launch");
     return VT_ATTN_OK;
@@ -132,7 +152,7 @@ extern "C" int vt_attn_accumulate_partial(float *acc, const void *part, long lon
     if (rc != VT_ATTN_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const __nv_bfloat16 *p = static_cast<const __nv_bfloat16 *>(part);
-    accumulate_kernel<<<merge_grid(n_rows, D), 256, 0, st>>>(acc, p, n_rows, D, first);
+    accumulate_kernel<<<merge_grid(n_rows, D / 8), 256, 0, st>>>(acc, p, n_rows, D, first);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "accumulate_kernel launch");
     return VT_ATTN_OK;

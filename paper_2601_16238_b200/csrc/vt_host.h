@@ -7,6 +7,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/vt_attn.h"
 #include "vt_ptx.cuh"
 

@@ -217,3 +217,82 @@ def test_forward_kernel_choice(lib):
     assert vt.vt_attn_fwd_kernel_kind(4, 16, 16, 1024, 1024, 128, False) == 0      # not causal
     assert vt.vt_attn_fwd_kernel_kind(4, 16, 16, 1024, 2048, 128, 2) == 0          # bottom-right with Sk != Sq
     assert vt.vt_attn_fwd_kernel_kind(4, 16, 16, 1024, 1024, 128, 2) == 2          # ... with Sk == Sq: the same mask
+
+
+# ------------------------------------------------------------------------------------------------
+# The binding checks every tensor's shape against the others before the library is entered (the kernels trust the sizes
+# they are told).  Shapes are checked before devices, so CPU tensors reach these checks without a GPU.
+# ------------------------------------------------------------------------------------------------
+def _t(*shape, dtype=None):
+    import torch
+    return torch.zeros(*shape, dtype=dtype or torch.bfloat16)
+
+
+@pytest.mark.parametrize("bad", ["v_short", "v_heads", "k_batch", "k_dim", "gqa", "o_shape", "lse_shape", "rank"])
+def test_forward_binding_rejects_mismatched_shapes(lib, bad):
+    import torch
+    q, k, v = _t(2, 4, 10, 64), _t(2, 2, 12, 64), _t(2, 2, 12, 64)
+    o = lse = None
+    if bad == "v_short":
+        v = _t(2, 2, 11, 64)
+    elif bad == "v_heads":
+        v = _t(2, 1, 12, 64)
+    elif bad == "k_batch":
+        k = _t(1, 2, 12, 64)
+    elif bad == "k_dim":
+        k = _t(2, 2, 12, 32)
+    elif bad == "gqa":
+        k, v = _t(2, 3, 12, 64), _t(2, 3, 12, 64)
+    elif bad == "o_shape":
+        o = _t(2, 4, 9, 64)
+    elif bad == "lse_shape":
+        lse = _t(2, 4, 9, dtype=torch.float32)
+    elif bad == "rank":
+        q = _t(2, 40, 64)
+    with pytest.raises(ValueError, match="shape|disagree|multiple|match|must be"):
+        vt.vt_attn_fwd(q, k, v, False, 0.125, o, lse)
+    if bad not in ("rank",):
+        with pytest.raises(ValueError, match="shape|disagree|multiple|match|must be"):
+            vt.vt_attn_fwd_splitkv(q, k, v, False, 0.125, 2, o, lse)
+
+
+@pytest.mark.parametrize("bad", ["o", "d_o", "lse", "dq", "dk", "dv", "v"])
+def test_backward_binding_rejects_mismatched_shapes(lib, bad):
+    import torch
+    q, k, v = _t(1, 4, 10, 64), _t(1, 2, 12, 64), _t(1, 2, 12, 64)
+    args = dict(o=_t(1, 4, 10, 64), d_o=_t(1, 4, 10, 64), lse=_t(1, 4, 10, dtype=torch.float32), dq=None, dk=None, dv=None)
+    wrong = {"o": _t(1, 4, 9, 64), "d_o": _t(1, 4, 10, 32), "lse": _t(1, 4, 11, dtype=torch.float32), "dq": _t(1, 4, 9, 64),
+             "dk": _t(1, 2, 11, 64), "dv": _t(1, 2, 12, 32)}
+    if bad == "v":
+        v = _t(1, 2, 13, 64)
+    else:
+        args[bad] = wrong[bad]
+    with pytest.raises(ValueError, match="shape|match"):
+        vt.vt_attn_bwd(q, k, v, args["o"], args["d_o"], args["lse"], True, 0.125, args["dq"], args["dk"], args["dv"])
+    full = {n: (t if t is not None else _t(*{"dq": q, "dk": k, "dv": v}[n].shape)) for n, t in args.items()}
+    if bad == "v":
+        full["dv"] = _t(1, 2, 12, 64)
+    with pytest.raises(ValueError, match="shape|match"):
+        vt.vt_attn_bwd_static_scratch(q, k, v, full["o"], full["d_o"], full["lse"], True, 0.125, full["dq"], full["dk"], full["dv"])
+
+
+def test_packed_and_host_bindings_reject_mismatched_shapes(lib):
+    import torch
+    q, k, v = _t(30, 4, 64), _t(40, 2, 64), _t(39, 2, 64)
+    cu = torch.tensor([0, 10, 30], dtype=torch.int32)
+    with pytest.raises(ValueError, match="shape"):
+        vt.vt_attn_fwd_varlen(q, k, v, cu, cu, 20, 20, True, 0.125)
+    v = _t(40, 2, 64)
+    with pytest.raises(ValueError, match="shape"):
+        vt.vt_attn_fwd_varlen(q, k, v, cu, cu, 20, 20, True, 0.125, lse=_t(30, 4, dtype=torch.float32))
+    with pytest.raises(ValueError, match="shape"):
+        vt.vt_attn_bwd_varlen(q, k, v, _t(30, 4, 64), _t(29, 4, 64), _t(4, 30, dtype=torch.float32), cu, cu, 20, 20, True, 0.125)
+    # host-buffer entry points: host tensors are what they take, so every check is reachable here
+    hq, hk, hv = _t(1, 2, 8, 64), _t(1, 2, 8, 64), _t(1, 2, 7, 64)
+    stage = torch.zeros(1024, dtype=torch.uint8)
+    with pytest.raises(ValueError, match="match"):
+        vt.vt_attn_fwd_host(hq, hk, hv, _t(1, 2, 8, 64), _t(1, 2, 8, dtype=torch.float32), False, 0.125, stage)
+    with pytest.raises(ValueError, match="shape"):
+        vt.vt_attn_fwd_host(hq, hk, hk, _t(1, 2, 9, 64), _t(1, 2, 8, dtype=torch.float32), False, 0.125, stage)
+    with pytest.raises(ValueError, match="shape"):
+        vt.vt_attn_merge_partial(_t(4, 64, dtype=torch.float32), _t(5, dtype=torch.float32), _t(4, 64), _t(4, dtype=torch.float32), True)

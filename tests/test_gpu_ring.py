@@ -29,6 +29,33 @@ def test_merge_of_key_blocks_equals_attention_over_all_keys(vt, D):
     assert (np.abs(host(lse_acc) - lse_ref) <= TOL_LSE * np.maximum(1.0, np.abs(lse_ref))).all()
 
 
+@pytest.mark.parametrize("D", [96, 192])
+def test_merge_of_many_rows_whose_threads_straddle_warps(vt, D):
+    """49 152 query rows at head dimensions whose D / 8 threads per row (12, 24) do not divide a warp: more blocks than the
+    GPU holds at once, so a thread of a row may run long after the row's first thread.  The merged result must still be
+    attention over all keys (every thread of a row has to weigh with the OLD running LSE), and the same bits every run."""
+    import torch
+    cfg = AttnConfig("merge_many", 18, 1, 3, 3, 16384, 192, D, False, False)
+    q, k, v = make_inputs(cfg, with_do=False)
+    tq, tk, tv = dev(q), dev(k), dev(v)
+    parts = [vt.vt_attn_fwd(tq, tk[:, :, a:a + 64].contiguous(), tv[:, :, a:a + 64].contiguous(), False, cfg.scale)
+             for a in (0, 64, 128)]
+    runs = []
+    for _ in range(3):
+        o_acc = torch.full(tq.shape, float("nan"), dtype=torch.float32, device="cuda")
+        lse_acc = torch.full(tq.shape[:3], float("nan"), dtype=torch.float32, device="cuda")
+        for i, (o_p, lse_p) in enumerate(parts):
+            vt.vt_attn_merge_partial(o_acc, lse_acc, o_p, lse_p, first=(i == 0))
+        runs.append((o_acc, lse_acc, vt.vt_attn_merge_finish(o_acc)))
+    torch.cuda.synchronize()
+    for o_acc, lse_acc, o in runs[1:]:
+        assert torch.equal(o_acc, runs[0][0]) and torch.equal(lse_acc, runs[0][1]) and torch.equal(o, runs[0][2])
+    o_ref, lse_ref = orc.attn_fwd(q, k, v, False, cfg.scale)
+    assert np.abs(host(runs[0][2]) - o_ref).max() <= TOL_O
+    assert np.abs(host(runs[0][0]) - o_ref).max() <= TOL_O
+    assert (np.abs(host(runs[0][1]) - lse_ref) <= TOL_LSE * np.maximum(1.0, np.abs(lse_ref))).all()
+
+
 def test_merge_with_empty_parts(vt):
     import torch
     n, D = 300, 64

@@ -189,6 +189,71 @@ def test_bounded_wait_reports_a_timeout_and_the_context_survives(vt):
     check_fwd(host(o), host(lse), o_ref, lse_ref, "after timeout")
 
 
+def test_status_word_without_synchronising(vt):
+    """The non-blocking pair: the copy of the status word is enqueued into pinned host memory and is valid once the caller
+    has synchronised; the reset is enqueued too."""
+    import torch
+    assert vt.vt_attn_device_status()[0] == 0
+    word = torch.full((1,), -1, dtype=torch.int32).pin_memory()
+    vt.vt_attn_device_status_async(word)
+    torch.cuda.synchronize()
+    assert int(word[0]) == 0
+    vt.vt_attn_selftest_timeout(20)
+    vt.vt_attn_device_status_async(word)
+    vt.vt_attn_device_status_clear()
+    torch.cuda.synchronize()
+    assert int(word[0]) & 0xFF == 9 and (int(word[0]) >> 8) & 0xFF == 3
+    assert vt.vt_attn_device_status()[0] == 0           # cleared by the enqueued reset
+
+
+def test_host_buffer_calls_from_two_threads(vt):
+    """Two host threads call the host-buffer forward + backward on their own streams and staging areas at the same
+    time; each must get the bits a lone call gives (the library's two side streams and their events are shared)."""
+    import threading
+    import torch
+    cfgs = [CONFIGS["minigpt"], CONFIGS["vit"].with_(B=16)]
+    jobs = []
+    for c in cfgs:
+        bits = make_inputs(c)
+        hq, hk, hv, hdo = (torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).view(torch.bfloat16).pin_memory() for x in bits)
+        outs = [torch.empty_like(hq).pin_memory(), torch.empty(hq.shape[:3], dtype=torch.float32).pin_memory(),
+                torch.empty_like(hq).pin_memory(), torch.empty_like(hk).pin_memory(), torch.empty_like(hv).pin_memory()]
+        staging = torch.empty(vt.vt_attn_host_staging_bytes(c.B, c.Hq, c.Hkv, c.Sq, c.Sk, c.D, True), dtype=torch.uint8, device="cuda")
+        jobs.append((c, (hq, hk, hv, hdo), outs, staging, torch.cuda.Stream()))
+
+    def run(job, rounds):
+        c, (hq, hk, hv, hdo), (o, lse, dq, dk, dv), staging, st = job
+        for _ in range(rounds):
+            vt.vt_attn_fwd_bwd_host(hq, hk, hv, hdo, o, lse, dq, dk, dv, c.causal, c.scale, staging, stream=st)
+        st.synchronize()
+
+    want = []
+    for job in jobs:                                     # serial reference
+        run(job, 1)
+        want.append([t.clone() for t in job[2]])
+        for t in job[2]:
+            t.zero_()
+    errors = []
+
+    def guarded(job):
+        try:
+            run(job, 25)
+        except Exception as e:                           # noqa: BLE001
+            errors.append(e)
+
+    threads = [threading.Thread(target=guarded, args=(job,)) for job in jobs]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    torch.cuda.synchronize()
+    assert not errors, errors
+    assert vt.vt_attn_device_status()[0] == 0
+    for job, w in zip(jobs, want):
+        for a, b in zip(job[2], w):
+            assert torch.equal(a, b)
+
+
 def test_calls_can_be_captured_in_a_cuda_graph(vt):
     """The entry points neither synchronise nor allocate, so a stream capture around them works and
     replays give the same bits."""

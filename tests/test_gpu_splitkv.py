@@ -123,3 +123,28 @@ def test_packed_splitkv_matches_the_oracle(vt, Hq, Hkv, D, causal, lens_q, lens_
     o1, lse1 = vt.vt_attn_fwd_varlen(tq, tk, tv, cq, ck, max(lens_q), max(lens_k), causal, scale)
     torch.cuda.synchronize()
     assert np.abs(o_h - host(o1)).max() <= 2.0 ** -7 * max(1.0, np.abs(o_ref).max())
+
+
+def test_packed_splitkv_with_max_sq_below_the_longest_sequence(vt):
+    """A max_sq that does not cover the longest sequence: its first max_sq tokens (rounded up to whole 128-row tiles) are
+    attended as usual, the tokens no block owns come out as O = 0, LSE = -inf - never as whatever the scratch held."""
+    import torch
+    from paper_2601_16238_b200.inputs import normal_bf16
+    Hq, Hkv, D, lens_q, lens_k = 4, 2, 64, [300, 40], [600, 500]
+    cu_q = np.concatenate([[0], np.cumsum(lens_q)]).astype(np.int32)
+    cu_k = np.concatenate([[0], np.cumsum(lens_k)]).astype(np.int32)
+    q, k, v = (normal_bf16(s, 8900 + i) for i, s in enumerate(((340, Hq, D), (1100, Hkv, D), (1100, Hkv, D))))
+    scale = 0.125
+    cq, ck = torch.from_numpy(cu_q).cuda(), torch.from_numpy(cu_k).cuda()
+    need = vt.load_library().vt_attn_fwd_splitkv_varlen_workspace_bytes(2, Hq, Hkv, 340, 128, 600, D, 3)
+    ws = torch.full((need // 4,), 1e30, dtype=torch.float32, device="cuda").view(torch.uint8)     # poisoned scratch
+    o, lse = vt.vt_attn_fwd_splitkv_varlen(dev(q), dev(k), dev(v), cq, ck, 128, 600, 0, scale, 3, workspace=ws)
+    torch.cuda.synchronize()
+    assert vt.vt_attn_device_status()[0] == 0
+    o_ref, lse_ref = orc.attn_fwd_varlen(q, k, v, cu_q, cu_k, 0, scale)
+    o_h, lse_h = host(o), host(lse)
+    done = np.r_[0:128, 300:340]                        # one tile of the long sequence, all of the short one
+    left = np.r_[128:300]
+    assert np.abs(o_h[done] - o_ref[done]).max() <= TOL_O
+    assert (np.abs(lse_h[:, done] - lse_ref[:, done]) <= TOL_LSE * np.maximum(1.0, np.abs(lse_ref[:, done]))).all()
+    assert (o_h[left] == 0.0).all() and np.isneginf(lse_h[:, left]).all()

@@ -308,11 +308,19 @@ def test_bad_shapes_rejected():
 
 
 def test_result_independent_of_thread_count():
-    q, k, v, do = rand(2, 4, 20, 8), rand(2, 2, 20, 8), rand(2, 2, 20, 8), rand(2, 4, 20, 8)
-    a = orc.attn_bwd(q, k, v, do, True, 0.3)
-    b = orc.attn_bwd(q, k, v, do, True, 0.3)
-    for x, y in zip(a, b):
-        np.testing.assert_array_equal(x, y)
+    """One thread against all cores (and an odd count in between): the same bits, forward and backward."""
+    q, k, v, do = rand(3, 4, 20, 8), rand(3, 2, 20, 8), rand(3, 2, 20, 8), rand(3, 4, 20, 8)
+    before = orc.num_threads()
+    try:
+        results = []
+        for n in (1, 3, max(2, before)):
+            assert orc.set_num_threads(n) == n
+            results.append(orc.attn_fwd(q, k, v, True, 0.3) + orc.attn_bwd(q, k, v, do, True, 0.3))
+    finally:
+        orc.set_num_threads(before)
+    for other in results[1:]:
+        for x, y in zip(results[0], other):
+            np.testing.assert_array_equal(x, y)
 
 
 # --------------------------------------------------------------------------- packed (variable-length) batches
@@ -444,3 +452,24 @@ def test_f16_bit_widening_is_exact():
     bits = np.array([0x3C00, 0xBC00, 0x7BFF, 0x0001, 0x3555, 0x0000, 0x0400], dtype=np.uint16)
     want = [1.0, -1.0, 65504.0, 2.0 ** -24, 0.333251953125, 0.0, 2.0 ** -14]
     np.testing.assert_array_equal(orc.f16_bits_to_f64(bits), np.array(want))
+
+
+# --------------------------------------------------------------------------- stored expected values
+def test_stored_gqa_long_group_agrees_with_the_oracle_where_it_is_cheap_to_recompute():
+    """tests/golden/gqa_long_group5.npz (written by tests/golden/make_gqa_long_golden.py from the oracle alone) against a
+    fresh oracle run on the part that needs no long computation: under the causal mask the first query tile sees only
+    the first 128 keys, so its O, LSE and dQ are those of the 128 x 128 causal problem."""
+    import os
+    from paper_2601_16238_b200.inputs import CONFIGS, make_inputs
+    gold = np.load(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "gqa_long_group5.npz"))
+    cfg = CONFIGS["gqa_long"]
+    g, G = int(gold["group"]), cfg.Hq // cfg.Hkv
+    assert list(gold["query_tiles"])[0] == 0 and gold["o"].shape == (G, 3 * 128, cfg.D) and gold["dk"].shape == (3 * 128, cfg.D)
+    q, k, v, d_o = make_inputs(cfg)
+    hs = slice(g * G, (g + 1) * G)
+    qs, ks, vs, dos = q[:, hs, :128], k[:, g:g + 1, :128], v[:, g:g + 1, :128], d_o[:, hs, :128]
+    o, lse = orc.attn_fwd(qs, ks, vs, True, cfg.scale)
+    dq, _, _ = orc.attn_bwd(qs, ks, vs, dos, True, cfg.scale)
+    np.testing.assert_allclose(gold["o"][:, :128], o[0], rtol=1e-6, atol=1e-7)
+    np.testing.assert_allclose(gold["lse"][:, :128], lse[0], rtol=1e-6, atol=1e-7)
+    np.testing.assert_allclose(gold["dq"][:, :128], dq[0], rtol=1e-6, atol=1e-7)
