@@ -59,6 +59,9 @@ NCU_TRAFFIC_BYTES = {
     # profiles/launch_lists.md, decoding: split-KV kernel 537.0 + 1.3 MB, merge kernel 0.6 MB per step
     "decode_32k": 538.9e6,
 }
+NCU_TRAFFIC_NOTE = {
+    "sdpa_s8192_nc": "scaled x2 from the S = 4096 capture of the same kernel",
+}
 
 
 def load_peaks():
@@ -204,9 +207,11 @@ def run_varlen(args):
     touched = 2 * qb + 2 * kvb + lse.numel() * 4 + ((3 * qb + 2 * kvb + lse.numel() * 4) + (qb + 2 * kvb) if with_bwd else 0)
     flush, l2_note = None, f"inputs+outputs {touched / 1e6:.0f} MB exceed the 126 MB L2"
     if touched <= 2 * L2_BYTES:
-        scratch = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
-        flush = lambda: scratch.fill_(1)      # noqa: E731
-        l2_note = "L2 flushed (252 MB write) before every timed step"
+        # flushed by READING a buffer twice the size of L2: a write flush would leave dirty lines whose write-back lands
+        # inside the timed kernels
+        scratch = torch.zeros(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
+        flush = lambda: scratch.max()      # noqa: E731
+        l2_note = "L2 flushed (252 MB read) before every timed step"
     with ClockSampler(local_rank) as clocks:
         ms = time_steps(torch, step, args.steps, args.warmup, flush)
     rc, detail = vt.vt_attn_device_status()
@@ -351,6 +356,59 @@ def run_decode_ragged(args):
     print(json.dumps(line), flush=True)
 
 
+def extra_fwd_bwd(torch, vt, peaks, local_rank, steps, warmup):
+    """The forward + backward half of the metric, timed in the same run: the long-context GQA configuration
+    (B = 1, 32 query heads on 8 KV heads, S = 16384, D = 128, causal), vt_attn_fwd followed by vt_attn_bwd."""
+    cfg = CONFIGS["gqa_long"]
+    q, k, v, d_o = device_tensors(cfg, torch, True)
+    o = torch.empty_like(q)
+    lse = torch.empty(q.shape[:3], dtype=torch.float32, device="cuda")
+    dq, dk, dv = torch.empty_like(q), torch.empty_like(k), torch.empty_like(v)
+    dims = (cfg.B, cfg.Hq, cfg.Hkv, cfg.Sq, cfg.Sk, cfg.D)
+    ws = torch.empty(max(256, vt.vt_attn_bwd_workspace_bytes(*dims)), dtype=torch.uint8, device="cuda")
+
+    def step():
+        vt.vt_attn_fwd(q, k, v, cfg.causal, cfg.scale, o, lse)
+        vt.vt_attn_bwd(q, k, v, o, d_o, lse, cfg.causal, cfg.scale, dq, dk, dv, ws)
+
+    def bwd_only():
+        vt.vt_attn_bwd(q, k, v, o, d_o, lse, cfg.causal, cfg.scale, dq, dk, dv, ws)
+
+    with ClockSampler(local_rank) as clocks:
+        ms = max_over_ranks(time_steps(torch, step, steps, warmup, None), device="cuda")
+    ms_bwd = max_over_ranks(time_steps(torch, bwd_only, steps, 1, None), device="cuda")
+    rc, detail = vt.vt_attn_device_status()
+    if rc != 0:
+        raise SystemExit(f"device status {rc} (detail {detail:#x}) after the forward + backward region")
+    flops = cfg.fwd_flops() * 3.5
+    tf = flops / (ms * 1e-3) / 1e12
+    tf_bwd = cfg.bwd_flops() / (ms_bwd * 1e-3) / 1e12
+    info = vt.vt_attn_get_info()
+    touched = algorithmic_bytes(cfg, "fwd_bwd")
+    return {"workload": cfg.name, "mode": "fwd_bwd", "ms_per_step": ms, "steps": steps, "warmup": warmup, "value": tf, "unit": "TFLOP/s",
+            "frac_of_measured_burst_peak": tf / float(peaks["bf16_tflops"]),
+            "frac_of_measured_sustained_peak": tf / float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])),
+            "frac_of_datasheet_peak": tf / DATASHEET_BF16_TFLOPS,
+            "backward_only": {"ms_per_step": ms_bwd, "value": tf_bwd, "frac_of_measured_burst_peak": tf_bwd / float(peaks["bf16_tflops"])},
+            "gpu_launches": (info[6] + info[7]) * steps, "l2": f"inputs+outputs {touched / 1e6:.0f} MB exceed the 126 MB L2",
+            "traffic": NCU_TRAFFIC_BYTES.get("gqa_long_bwd"), "algorithmic_bytes": int(touched), "clocks": clocks.summary()}
+
+
+def extra_sustained(torch, step, flops, peaks, local_rank, ms_hint, seconds=2.5):
+    """The default workload back to back for at least `seconds` of device time (the power cap pulls the SM clock down
+    after a few hundred milliseconds), with the median SM clock sampled meanwhile: time x MHz shows how the number
+    depends on the clock without touching any setting."""
+    n = max(20, int(seconds * 1e3 / max(ms_hint, 1e-3)) + 1)
+    with ClockSampler(local_rank) as clocks:
+        ms = max_over_ranks(time_steps(torch, step, n, 3, None), device="cuda")
+    tf = flops / (ms * 1e-3) / 1e12
+    c = clocks.summary()
+    return {"steps": n, "ms_per_step": ms, "timed_seconds": n * ms * 1e-3, "value": tf, "unit": "TFLOP/s",
+            "frac_of_measured_sustained_peak": tf / float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])),
+            "frac_of_measured_burst_peak": tf / float(peaks["bf16_tflops"]),
+            "ms_times_sm_mhz": (ms * c["sm_mhz"]) if c["sm_mhz"] else None, "clocks": c}
+
+
 def run_ours(args):
     import torch
     import paper_2601_16238_b200 as vt
@@ -403,9 +461,11 @@ def run_ours(args):
     flush = None
     l2_note = f"inputs+outputs {touched / 1e6:.0f} MB exceed the 126 MB L2"
     if touched <= 2 * L2_BYTES:
-        scratch = torch.empty(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
-        flush = lambda: scratch.fill_(1)      # noqa: E731
-        l2_note = "L2 flushed (252 MB write) before every timed step"
+        # flushed by READING a buffer twice the size of L2: a write flush would leave dirty lines whose write-back lands
+        # inside the timed kernels
+        scratch = torch.zeros(2 * L2_BYTES, dtype=torch.uint8, device="cuda")
+        flush = lambda: scratch.max()      # noqa: E731
+        l2_note = "L2 flushed (252 MB read) before every timed step"
 
     info = vt.vt_attn_get_info()
     launches_per_step = 2 if use_split else info[6] + (info[7] if with_bwd else 0)      # split: chunk kernel + merge
@@ -430,9 +490,19 @@ def run_ours(args):
     tflops_per_gpu = flops / (ms * 1e-3) / 1e12
     value = tflops_per_gpu * world
 
+    # ---- the default line also carries the forward + backward half of the metric and a sustained figure
+    extras = {}
+    if args.workload == "sdpa_s8192_nc" and mode == "fwd" and not f16 and not args.lean:
+        burst_clocks = clocks.summary()
+        extras["sustained"] = extra_sustained(torch, timed_step, flops, peaks, local_rank, ms)
+        extras["sustained"]["burst_ms_times_sm_mhz"] = (ms * burst_clocks["sm_mhz"]) if burst_clocks["sm_mhz"] else None
+        torch.cuda.synchronize()
+        time.sleep(1.0)                      # let the clock recover before the next burst-sized region
+        extras["fwd_bwd"] = extra_fwd_bwd(torch, vt, peaks, local_rank, max(5, min(args.steps, 20)), 3)
+
     # ---- end to end through the host-buffer entry point: pinned host -> device -> kernels -> host
     e2e = None
-    if rank == 0 or world > 1:
+    if (rank == 0 or world > 1) and not args.lean:
         hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
         ho, hlse = torch.empty_like(hq).pin_memory(), torch.empty(lse.shape, dtype=torch.float32).pin_memory()
         staging = torch.empty(vt.vt_attn_host_staging_bytes(*dims, with_bwd), dtype=torch.uint8, device="cuda")
@@ -509,7 +579,13 @@ def run_ours(args):
         "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": launches_per_step * args.steps,
         "roofline": roofline,
     }
-    if world == 1 and not args.no_cpu_baseline:
+    if NCU_TRAFFIC_NOTE.get(cfg.name):
+        roofline["traffic_note"] = NCU_TRAFFIC_NOTE[cfg.name]
+    for key, val in extras.items():
+        if world > 1:
+            val = dict(val, value=val["value"] * world, note=f"whole job: {world} ranks, each the same per-GPU work")
+        line[key] = val
+    if world == 1 and not args.no_cpu_baseline and not args.lean:
         line["cpu_baseline"] = cpu_baseline(cfg, with_bwd, budget_s=args.cpu_budget)
     print(json.dumps(line), flush=True)
 
@@ -816,6 +892,9 @@ def main():
     ap.add_argument("--graph", action="store_true",
                     help="time replays of a CUDA graph holding one step's kernels (small workloads: takes the host's per-call work out)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--lean", action="store_true",
+                    help="only the timed region: no end-to-end leg, no forward+backward / sustained extras, no CPU baseline (the "
+                         "command line profiler captures run)")
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle work for the cpu_baseline object")
     ap.add_argument("--ref-budget", type=float, default=150.0, help="seconds the whole --impl reference run may take")
     args = ap.parse_args()
