@@ -50,18 +50,20 @@ L2_BYTES = 126 * 1024 * 1024
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of one launch of the dominant
 # kernel, from the ncu captures summarised under profiles/; None where no capture exists.
 NCU_TRAFFIC_BYTES = {
+    # profiles/attn_fwd_pair_kernel_sdpa_s8192_nc.md: 402.7 MB read + 115.0 MB written, one launch at full size
+    "sdpa_s8192_nc": 517.7e6,
     # profiles/attn_fwd_pair_kernel_sdpa_s4096_nc.md: 201.4 MB read + 50.0 MB written per launch
     "sdpa_s4096_nc": 251.4e6,
-    # the same capture scaled by the rows per head (2x): per-row traffic is the same, K/V re-reads stay in L2
-    "sdpa_s8192_nc": 502.8e6,
     # profiles/attn_fwd_kernel_paper_shape.md: 504.0 MB read + 156.3 MB written
     "paper_shape": 660.3e6,
     # profiles/launch_lists.md, decoding: split-KV kernel 537.0 + 1.3 MB, merge kernel 0.6 MB per step
     "decode_32k": 538.9e6,
+    # profiles/bwd_kernels_gqa_long.md, one launch of each kernel at full size: forward 312.3 MB; backward
+    # (Delta 273.9 + dK/dV 397.4 + dQ 454.0 MB)
+    "gqa_long": 312.3e6,
+    "gqa_long_bwd": 1125.3e6,
 }
-NCU_TRAFFIC_NOTE = {
-    "sdpa_s8192_nc": "scaled x2 from the S = 4096 capture of the same kernel",
-}
+NCU_TRAFFIC_NOTE = {}
 
 
 def load_peaks():
@@ -391,7 +393,9 @@ def extra_fwd_bwd(torch, vt, peaks, local_rank, steps, warmup):
             "frac_of_datasheet_peak": tf / DATASHEET_BF16_TFLOPS,
             "backward_only": {"ms_per_step": ms_bwd, "value": tf_bwd, "frac_of_measured_burst_peak": tf_bwd / float(peaks["bf16_tflops"])},
             "gpu_launches": (info[6] + info[7]) * steps, "l2": f"inputs+outputs {touched / 1e6:.0f} MB exceed the 126 MB L2",
-            "traffic": NCU_TRAFFIC_BYTES.get("gqa_long_bwd"), "algorithmic_bytes": int(touched), "clocks": clocks.summary()}
+            "traffic": {"forward_kernel": NCU_TRAFFIC_BYTES.get("gqa_long"), "backward_kernels": NCU_TRAFFIC_BYTES.get("gqa_long_bwd"),
+                        "source": "one ncu capture of each kernel at full size (profiles/bwd_kernels_gqa_long.md)"},
+            "algorithmic_bytes": int(touched), "clocks": clocks.summary()}
 
 
 def extra_sustained(torch, step, flops, peaks, local_rank, ms_hint, seconds=2.5):
@@ -409,12 +413,153 @@ def extra_sustained(torch, step, flops, peaks, local_rank, ms_hint, seconds=2.5)
             "ms_times_sm_mhz": (ms * c["sm_mhz"]) if c["sm_mhz"] else None, "clocks": c}
 
 
+# ------------------------------------------------------------------------------------------------
+# Context-parallel ring attention: one causal sequence sharded over the ranks in the zig-zag layout, forward + backward.
+# The one workload with a real exchange step (K / V blocks and the running dK / dV travel around the ring with
+# torch.distributed point-to-point operations: NCCL on GPUs); total work is fixed, so scaling is "strong".
+# ------------------------------------------------------------------------------------------------
+RING_WORKLOADS = {
+    # name: B, Hq, Hkv, S (whole sequence), D; the sequence is generated in 16 seeded pieces so that every world size
+    # (1, 2, 4, 8) sees the same data
+    "ring_causal_64k": {"B": 1, "Hq": 32, "Hkv": 8, "S": 65536, "D": 128, "pieces": 16, "index": 31},
+}
+
+
+def ring_shard_bits(w, rank, world):
+    """This rank's zig-zag shard of the workload's seeded inputs: four uint16 arrays [2, B, H, S_chunk, D] (q, k, v, dO)."""
+    from paper_2601_16238_b200.inputs import normal_bf16
+    from paper_2601_16238_b200.ring import zigzag_chunks
+    if w["pieces"] % (2 * world) != 0:
+        raise SystemExit(f"world size {world}: 2 * world must divide {w['pieces']}")
+    per_chunk = w["pieces"] // (2 * world)
+    rows = w["S"] // w["pieces"]
+    out = []
+    for t, heads in enumerate((w["Hq"], w["Hkv"], w["Hkv"], w["Hq"])):
+        chunks = []
+        for c in zigzag_chunks(rank, world):
+            pieces = [normal_bf16((w["B"], heads, rows, w["D"]), 1000 * w["index"] + 100 * t + piece)
+                      for piece in range(c * per_chunk, (c + 1) * per_chunk)]
+            chunks.append(np.concatenate(pieces, axis=2))
+        out.append(np.stack(chunks))
+    return out
+
+
+def ring_step(q2, k2, v2, do2, scale, group=None, comm_stream=None, **standins):
+    """One step of the ring workload on this rank: causal forward + backward in the zig-zag layout."""
+    from paper_2601_16238_b200.ring import ring_attention_zigzag_fwd_bwd
+    return ring_attention_zigzag_fwd_bwd(q2, k2, v2, do2, scale, group, comm_stream, **standins)
+
+
+def run_ring(args):
+    import torch
+    import paper_2601_16238_b200 as vt
+    from paper_2601_16238_b200 import ring as ring_mod
+
+    w = RING_WORKLOADS[args.workload]
+    rank, local_rank, world = env_rank_world()
+    torch.cuda.set_device(local_rank)
+    init_process_group("nccl")
+    vt.load_library()
+    peaks, peak_kind = load_peaks()
+    scale = float(np.float32(1.0) / np.sqrt(np.float32(w["D"])))
+    bits = ring_shard_bits(w, rank, world)
+    q2, k2, v2, do2 = (torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).cuda() for x in bits)
+    comm = torch.cuda.Stream() if world > 1 else None
+    info = vt.vt_attn_get_info()
+    launches = [0]
+
+    def attend(q, k, v, mode, sc):                       # the library's kernels, counted
+        launches[0] += info[6]
+        return vt.vt_attn_fwd(q, k, v, mode, sc)
+
+    def attend_bwd(q, k, v, o, d_o, lse, mode, sc):
+        launches[0] += info[7]
+        return vt.vt_attn_bwd(q, k, v, o, d_o, lse, mode, sc)
+
+    class Merge(ring_mod._DeviceMerge):
+        def add(self, o_part, lse_part):
+            launches[0] += 1
+            super().add(o_part, lse_part)
+
+        def result(self):
+            launches[0] += 1
+            return super().result()
+
+    class Sum(ring_mod._DeviceSum):
+        def add(self, part):
+            launches[0] += 1
+            super().add(part)
+
+        def result(self):
+            launches[0] += 1
+            return super().result()
+
+    outs = [None]
+
+    def step():
+        outs[0] = ring_step(q2, k2, v2, do2, scale, None, comm, attend=attend, merge_factory=Merge, attend_bwd=attend_bwd, sum_factory=Sum)
+
+    with ClockSampler(local_rank) as clocks:
+        ms = max_over_ranks(time_steps(torch, step, args.steps, args.warmup, None), device="cuda")
+    per_step_launches = launches[0] // (args.steps + args.warmup)
+    rc, detail = vt.vt_attn_device_status()
+    if rc != 0:
+        raise SystemExit(f"device status {rc} (detail {detail:#x}) after the timed region")
+    flops = 4.0 * w["B"] * w["Hq"] * float(w["S"]) ** 2 * w["D"] * 0.5 * 3.5
+    tflops = flops / (ms * 1e-3) / 1e12
+
+    # end to end: this rank's shards start in pinned host memory, its results end there
+    host_in = [t.cpu().pin_memory() for t in (q2, k2, v2, do2)]
+    host_out = [torch.empty_like(t, device="cpu").pin_memory() for t in outs[0]]
+
+    def e2e_step():
+        for h, d in zip(host_in, (q2, k2, v2, do2)):
+            d.copy_(h, non_blocking=True)
+        step()
+        for h, d in zip(host_out, outs[0]):
+            h.copy_(d, non_blocking=True)
+    e2e_steps = max(3, min(args.steps, 5))
+    e2e_ms = max_over_ranks(time_steps(torch, e2e_step, e2e_steps, 3, None), device="cuda")
+    if rank != 0:
+        return
+    peak = float(peaks["bf16_tflops"])
+    shard_bytes = sum(t.numel() * t.element_size() for t in (k2, v2))
+    line = {
+        "metric": "fused attention fwd+bwd TFLOP/s (bf16)", "value": tflops, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "B": w["B"], "Hq": w["Hq"], "Hkv": w["Hkv"], "S": w["S"], "D": w["D"], "causal": True,
+                   "mode": "fwd_bwd", "layout": f"zig-zag: rank r holds chunks r and {2 * world - 1} - r of {2 * world}",
+                   "exchange": "none (one rank)" if world == 1 else
+                               f"torch.distributed point-to-point (NCCL) on its own stream: {shard_bytes / 1e6:.1f} MB of K/V per step forward, "
+                               f"that plus {2 * shard_bytes / 1e6:.1f} MB of fp32 dK/dV sums per step backward",
+                   "l2": "inputs exceed the 126 MB L2", "flops_convention": "4*B*Hq*S^2*D*0.5 forward, backward 2.5x",
+                   "parallelism": f"cp{world} (sequence shards, ring exchange)"},
+        "pct_of_measured_bf16_peak": 100.0 * tflops / (peak * world), "clocks": clocks.summary(),
+        "e2e": {"value": flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host_in)) * world,
+                "d2h_bytes_per_step": int(sum(t.numel() * t.element_size() for t in host_out)) * world, "steps": e2e_steps,
+                "api": "pinned copies + ring_attention_zigzag_fwd_bwd"},
+        "gpu_launches": per_step_launches * args.steps,
+        "roofline": {"bound": "tensor", "kernel": "forward / backward attention kernels per block + merge and accumulate kernels",
+                     "achieved": tflops / world, "peak": peak, "unit": "TFLOP/s", "frac": tflops / world / peak,
+                     "peak_kind": f"{peak_kind} cuBLAS bf16 burst, per GPU", "traffic": None},
+    }
+    if world == 1 and not args.no_cpu_baseline and not args.lean:
+        from paper_2601_16238_b200.inputs import AttnConfig
+        cfg = AttnConfig(args.workload, w["index"], w["B"], w["Hq"], w["Hkv"], w["S"], w["S"], w["D"], True, True)
+        line["cpu_baseline"] = cpu_baseline(cfg, True, budget_s=args.cpu_budget)
+    print(json.dumps(line), flush=True)
+
+
 def run_ours(args):
     import torch
     import paper_2601_16238_b200 as vt
 
     if args.workload in VARLEN_CONFIGS:
         return run_varlen(args)
+    if args.workload in RING_WORKLOADS:
+        return run_ring(args)
     if args.workload == "decode_ragged":
         return run_decode_ragged(args)
 
@@ -658,7 +803,13 @@ def run_reference(args):
         return
     if args.workload in VARLEN_CONFIGS or args.workload == "decode_ragged":
         raise SystemExit("--impl reference covers the fixed-length workloads; packed ones report the oracle as cpu_baseline")
-    cfg = CONFIGS[args.workload]
+    if args.workload in RING_WORKLOADS:          # the oracle knows no ranks: the whole causal sequence, forward + backward
+        from paper_2601_16238_b200.inputs import AttnConfig
+        w = RING_WORKLOADS[args.workload]
+        cfg = AttnConfig(args.workload, w["index"], w["B"], w["Hq"], w["Hkv"], w["S"], w["S"], w["D"], True, True)
+        args.mode = "fwd_bwd"
+    else:
+        cfg = CONFIGS[args.workload]
     mode = args.mode or "fwd"
     with_bwd = mode == "fwd_bwd"
     from oracle import attn_oracle as orc
@@ -883,7 +1034,7 @@ def main():
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", default="sdpa_s8192_nc", choices=sorted(CONFIGS) + sorted(VARLEN_CONFIGS) + sorted(SUITE_WORKLOADS) + ["decode_ragged"])
+    ap.add_argument("--workload", default="sdpa_s8192_nc", choices=sorted(CONFIGS) + sorted(VARLEN_CONFIGS) + sorted(SUITE_WORKLOADS) + sorted(RING_WORKLOADS) + ["decode_ragged"])
     ap.add_argument("--mode", choices=["fwd", "fwd_bwd"], default=None)
     ap.add_argument("--splitkv", choices=["auto", "on", "off"], default="auto",
                     help="forward through vt_attn_fwd_splitkv: auto = when the library's plan splits the keys or packs a KV group's heads")

@@ -90,11 +90,49 @@ int vt_attn_fwd(const void *q, const void *k, const void *v,
                 int causal, float scale, void *stream);
 
 /*
+ * vt_attn_fwd with the rotary position embedding of the QUERIES applied inside the kernel
+ * (the paper's kernel microbenchmark table has "Rotary (fwd)" as a row of its own; this takes
+ * the query half of that operator into the attention kernel's load path, saving its pass
+ * over Q in global memory).  q is unrotated; every query tile is rotated in shared memory, in
+ * fp32 and rounded to bf16, before the first product: "rotate-half" convention, element i of a
+ * head pairs with element i + D/2, query i of the sequence sits at position q_pos0 + i:
+ *     q'[i] = q[i] cos[pos][i] - q[i + D/2] sin[pos][i],   q'[i + D/2] = q[i + D/2] cos[pos][i] + q[i] sin[pos][i]
+ * k_rotated must hold the ALREADY rotated keys (vt_suite_rope_apply): a key tile is read by
+ * every query tile of its head, rotating it inside the kernel would repeat the work each time.
+ * rope_cos, rope_sin: float [rope_positions, D/2] (vt_suite_rope_tables), device, 16-byte
+ * aligned; q_pos0 + Sq <= rope_positions.  D must be 64 or 128.  Everything else as vt_attn_fwd.
+ */
+int vt_attn_fwd_rope(const void *q, const void *k_rotated, const void *v,
+                     const float *rope_cos, const float *rope_sin,
+                     void *o, float *lse,
+                     int B, int Hq, int Hkv, int Sq, int Sk, int D,
+                     int causal, float scale, int q_pos0, int rope_positions, void *stream);
+
+/*
  * Bytes of device scratch vt_attn_bwd needs for this shape (0 on an invalid shape).
- * The scratch holds Delta[b,h,i] = sum_d dO*O in fp32.  Its contents on entry are
- * ignored; every word that is read is written first by the same call.
+ * The scratch holds Delta[b,h,i] = sum_d dO*O in fp32 and, for the shapes that take the
+ * single-pass backward (vt_attn_bwd_kernel_kind), a 32-bit accumulator per element of dQ
+ * plus a few per-head scalars.  Its contents on entry are ignored; every word that is
+ * read is written first by the same call.
  */
 size_t vt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int Sq, int Sk, int D);
+
+/*
+ * Which kernels vt_attn_bwd runs for a shape when it is given the workspace size stated
+ * above (host-only, launches nothing; a negative VT_ATTN_ERR_* for an invalid shape):
+ *   0  three kernels: Delta, then one kernel per key tile for dK / dV and one per query tile
+ *      for dQ; each output tile has one owner block (7 tile products per tile pair);
+ *   1  the single-pass backward, built for 64 < D <= 128: one kernel per key tile forms dK,
+ *      dV and that tile's share of dQ (5 tile products per tile pair); the shares are summed
+ *      in 32-bit fixed point, scaled per (batch, head) from bounds on dO, K and V, so the sum
+ *      does not depend on the order in which the blocks add and dQ is the same bits on every
+ *      run; a last pass rounds it to the tensors' type.  Six kernels and one memset per call.
+ * The library itself always answers 0: on the B200 the reductions of 1 cost more than the two
+ * products they save.  The environment variable VT_ATTN_BWD_PATH=fused (read at every call)
+ * selects 1 wherever it is built, for measurements and tests; =split or unset selects 0.  A
+ * call whose workspace only holds Delta (vt_attn_bwd_static_scratch does this) takes 0 too.
+ */
+int vt_attn_bwd_kernel_kind(int B, int Hq, int Hkv, int Sq, int Sk, int D);
 
 /*
  * Backward pass ("Attention (bwd)" row of the same table).  With P recomputed from
@@ -109,9 +147,10 @@ size_t vt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int Sq, int Sk, int D
  * q, k, v, o, d_o (bf16) and lse (float) are read only; o and lse must be the
  * outputs of vt_attn_fwd on the same q, k, v, causal and scale.
  * dq [B,Hq,Sq,D], dk and dv [B,Hkv,Sk,D] (bf16) are fully overwritten; every sum
- * is taken in a fixed order, so repeated calls give bit-identical results.
+ * is taken in a fixed order or in integer arithmetic, so repeated calls give
+ * bit-identical results.
  * workspace: device scratch of at least vt_attn_bwd_workspace_bytes(...) bytes,
- * 16-byte aligned, owned by the caller, not shared with a concurrent call.
+ * 256-byte aligned, owned by the caller, not shared with a concurrent call.
  */
 int vt_attn_bwd(const void *q, const void *k, const void *v,
                 const void *o, const void *d_o, const float *lse,

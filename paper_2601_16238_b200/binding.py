@@ -31,12 +31,14 @@ EXPORTS = {
     "vt_attn_status_string": (ctypes.c_char_p, [_i]),
     "vt_attn_last_cuda_error": (ctypes.c_char_p, []),
     "vt_attn_fwd": (_i, [_vp] * 5 + _DIMS + [_i, _f, _vp]),
+    "vt_attn_fwd_rope": (_i, [_vp] * 7 + _DIMS + [_i, _f, _i, _i, _vp]),
     "vt_attn_fwd_dv": (_i, [_vp] * 5 + _DIMS + [_i, _i, _f, _vp]),
     "vt_attn_fwd_dv_f16": (_i, [_vp] * 5 + _DIMS + [_i, _i, _f, _vp]),
     "vt_attn_fwd_kernel_kind": (_i, _DIMS + [_i]),
     "vt_attn_fwd_f16": (_i, [_vp] * 5 + _DIMS + [_i, _f, _vp]),
     "vt_attn_bwd_f16": (_i, [_vp] * 9 + _DIMS + [_i, _f, _vp, _sz, _vp]),
     "vt_attn_bwd_workspace_bytes": (_sz, _DIMS),
+    "vt_attn_bwd_kernel_kind": (_i, _DIMS),
     "vt_attn_bwd": (_i, [_vp] * 9 + _DIMS + [_i, _f, _vp, _sz, _vp]),
     "vt_attn_bwd_static_scratch": (_i, [_vp] * 9 + _DIMS + [_i, _f, _vp]),
     "vt_attn_bwd_static_scratch_f16": (_i, [_vp] * 9 + _DIMS + [_i, _f, _vp]),
@@ -197,6 +199,25 @@ def vt_attn_fwd(q, k, v, causal: bool, scale: float, o=None, lse=None, stream=No
     return _fwd("vt_attn_fwd", torch.bfloat16, q, k, v, causal, scale, o, lse, stream)
 
 
+def vt_attn_fwd_rope(q, k_rotated, v, rope_cos, rope_sin, causal, scale: float, q_pos0: int = 0, o=None, lse=None, stream=None):
+    """vt_attn_fwd with the rotary embedding of the queries applied inside the kernel: q unrotated, k_rotated already
+    rotated; rope_cos / rope_sin fp32 [positions, D/2].  Returns (O bf16, LSE fp32)."""
+    import torch
+    lib = load_library()
+    dims = _dims(q, k_rotated, v)
+    half = dims[5] // 2
+    if rope_cos.dim() != 2 or int(rope_cos.shape[1]) != half or rope_sin.shape != rope_cos.shape:
+        raise ValueError(f"rope_cos / rope_sin: expected [positions, {half}] tensors of the same shape")
+    o, lse = _outputs_fwd(q, o, lse, q.shape, q.shape[:3])
+    _inputs(torch.bfloat16, "cuda", q, k=k_rotated, v=v)
+    _require(rope_cos, torch.float32, "rope_cos", device=q.device)
+    _require(rope_sin, torch.float32, "rope_sin", device=q.device)
+    rc = _call(q.device, lib.vt_attn_fwd_rope, _p(q), _p(k_rotated), _p(v), _p(rope_cos), _p(rope_sin), _p(o), _p(lse), *dims,
+               _mask_mode(causal), float(scale), int(q_pos0), int(rope_cos.shape[0]), _stream(stream, q.device))
+    _check(rc, "vt_attn_fwd_rope")
+    return o, lse
+
+
 def _fwd_dv(name, dtype, q, k, v, causal, scale, o, lse, stream):
     lib = load_library()
     dims = _dims(q, k, v, own_dv=True)
@@ -239,6 +260,15 @@ def vt_attn_fwd_f16(q, k, v, causal: bool, scale: float, o=None, lse=None, strea
 
 def vt_attn_bwd_workspace_bytes(B, Hq, Hkv, Sq, Sk, D) -> int:
     return int(load_library().vt_attn_bwd_workspace_bytes(B, Hq, Hkv, Sq, Sk, D))
+
+
+def vt_attn_bwd_kernel_kind(B, Hq, Hkv, Sq, Sk, D) -> int:
+    """0: Delta + one kernel for dK / dV + one for dQ; 1: the single-pass backward (one kernel forms dK, dV and adds its
+    share of dQ into a fixed-point accumulator, a last pass rounds dQ)."""
+    rc = load_library().vt_attn_bwd_kernel_kind(B, Hq, Hkv, Sq, Sk, D)
+    if rc < 0:
+        _check(rc, "vt_attn_bwd_kernel_kind")
+    return rc
 
 
 def vt_attn_fwd_splitkv_plan(B, Hq, Hkv, Sq, Sk, D, n_splits=0):

@@ -15,6 +15,8 @@
 // Block = 384 threads: warp 0 and warp 2 TMA producers, warp 1 MMA issuer, warps 4..7 and 8..11 compute.
 // Recomputing S and dP in both kernels costs 7 tile products instead of 5 but every dQ, dK, dV tile has exactly
 // one owner block: no cross-block reduction, bit-identical results every run.
+#include <stdlib.h>
+
 #include <mutex>
 
 #include "vt_host.h"
@@ -815,6 +817,12 @@ bwd_dq_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ 
     }
 }
 
+}  // namespace vt
+
+#include "bwd_fused.cuh"
+
+namespace vt {
+
 template <typename K>
 static int set_smem(K kernel, int bytes, const char *what)
 {
@@ -877,14 +885,132 @@ static int launch_bwd(const BwdMaps &m, BwdParams prm, const __nv_bfloat16 *o, c
     return VT_ATTN_OK;
 }
 
+// ----------------------------------------------------------------------------------------------
+// The five-product path (bwd_fused.cuh): workspace layout, when it is used, launches
+// ----------------------------------------------------------------------------------------------
+static size_t align256(size_t x) { return (x + 255) & ~static_cast<size_t>(255); }
+
+struct FusedPlan {
+    size_t delta, acc, stats_do, stats_k, stats_v, qscale, total;     // byte offsets into the workspace; acc .. stats_v are cleared together
+    size_t clear_bytes;
+};
+
+static FusedPlan fused_plan(int B, int Hq, int Hkv, int Sq, int d)
+{
+    FusedPlan f;
+    const size_t rows = static_cast<size_t>(B) * Hq * Sq;
+    size_t off = 0;
+    auto take = [&off](size_t bytes) { const size_t at = off; off += align256(bytes); return at; };
+    f.delta = take(rows * 4);
+    f.acc = take(rows * d * 4);
+    f.stats_do = take(static_cast<size_t>(B) * Hq * 4);
+    f.stats_k = take(static_cast<size_t>(B) * Hkv * 4);
+    f.stats_v = take(static_cast<size_t>(B) * Hkv * 4);
+    f.clear_bytes = off - f.acc;
+    f.qscale = take(static_cast<size_t>(B) * Hq * 4);
+    f.total = off;
+    return f;
+}
+
+// 0: library's choice; 1: always the two-kernel path; 2: the five-product path wherever it is built (D in (64, 128],
+// batched layout).  Read from the environment variable VT_ATTN_BWD_PATH ("split" / "fused") at every call: a switch for
+// tests and measurements, not part of the ABI.
+static int bwd_path_override()
+{
+    const char *e = getenv("VT_ATTN_BWD_PATH");
+    if (!e) return 0;
+    if (e[0] == 's') return 1;
+    if (e[0] == 'f') return 2;
+    return 0;
+}
+
+// Whether vt_attn_bwd uses the five-product path for this shape (given a workspace of the size
+// vt_attn_bwd_workspace_bytes states).  It is built for the 128-column kernels.  The library never picks it by itself:
+// measured on the B200 it is slower than the two-kernel path on every shape tried (B = 1, 32 query heads on 8 KV heads,
+// S = 16384, causal: 13.2 ms against 6.2 ms; with the red.add instructions compiled out 5.1 ms) - 64 KB of reductions
+// per (query tile, key tile) pair is more than the L2 takes per SM in the time the five products need (a loop of nothing
+// but these reductions on all SMs: 3.2 TB/s into HBM-resident tiles, 5.5 TB/s into tiles four blocks share).
+static bool fused_wanted(int B, int Hq, int Hkv, int Sq, int Sk, int D)
+{
+    (void)B; (void)Hq; (void)Hkv; (void)Sq; (void)Sk;
+    if (padded_head_dim(D) != 128) return false;
+    return bwd_path_override() == 2;
+}
+
+template <bool CAUSAL, bool F16>
+static int launch_bwd_fused(const BwdMaps &m, BwdParams prm, const __nv_bfloat16 *o, const __nv_bfloat16 *d_o, const __nv_bfloat16 *k,
+                            const __nv_bfloat16 *v, uint8_t *ws, int B, cudaStream_t stream)
+{
+    constexpr int D = 128;
+    int rc;
+    static std::atomic<bool> configured[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (!configured[dev & 63].load(std::memory_order_acquire)) {
+        if ((rc = set_smem(bwd_fused_kernel<D, CAUSAL, F16>, FusedSmem<D>::BYTES, "cudaFuncSetAttribute(fused)")) != VT_ATTN_OK) return rc;
+        configured[dev & 63].store(true, std::memory_order_release);
+    }
+    const FusedPlan f = fused_plan(B, prm.Hq, prm.Hkv, prm.Sq, prm.d);
+    float *delta = reinterpret_cast<float *>(ws + f.delta);
+    int *acc = reinterpret_cast<int *>(ws + f.acc);
+    float *stats_do = reinterpret_cast<float *>(ws + f.stats_do), *stats_k = reinterpret_cast<float *>(ws + f.stats_k);
+    float *stats_v = reinterpret_cast<float *>(ws + f.stats_v), *qscale = reinterpret_cast<float *>(ws + f.qscale);
+    cudaError_t e = cudaMemsetAsync(acc, 0, f.clear_bytes, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync(dQ accumulator)");
+
+    const long long n_rows = static_cast<long long>(B) * prm.Hq * prm.Sq;
+    const long long n_kv_rows = static_cast<long long>(B) * prm.Hkv * prm.Sk;
+    int tpr = 1;
+    while (tpr * 8 < prm.d) tpr *= 2;
+    const int rows_per_block = 256 / tpr;
+    long long delta_blocks = (n_rows + rows_per_block - 1) / rows_per_block;
+    if (delta_blocks > NUM_SMS * 32) delta_blocks = NUM_SMS * 32;
+    const int db = static_cast<int>(delta_blocks);
+    if (tpr == 16) bwd_delta_kernel<16, F16><<<db, 256, 0, stream>>>(o, d_o, delta, n_rows, 0, prm.d);
+    else bwd_delta_kernel<8, F16><<<db, 256, 0, stream>>>(o, d_o, delta, n_rows, 0, prm.d);      // 64 < d <= 128: tpr is 16 (d > 64)
+    if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_delta_kernel launch");
+    auto warp_grid = [](long long rows) { long long nb = (rows + 7) / 8; return static_cast<int>(nb > NUM_SMS * 16 ? NUM_SMS * 16 : nb); };
+    bwd_do_norm_kernel<F16><<<warp_grid(n_rows), 256, 0, stream>>>(d_o, stats_do, prm.Sq, prm.d, n_rows);
+    if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_do_norm_kernel launch");
+    bwd_kv_norm_kernel<F16><<<warp_grid(n_kv_rows), 256, 0, stream>>>(k, v, stats_k, stats_v, prm.Sk, prm.d, n_kv_rows);
+    if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_kv_norm_kernel launch");
+    const int n_bh = B * prm.Hq;
+    bwd_qscale_kernel<<<(n_bh + 127) / 128, 128, 0, stream>>>(stats_do, stats_k, stats_v, qscale, n_bh, prm.Hq, prm.Hkv);
+    if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_qscale_kernel launch");
+
+    prm.delta = delta;
+    prm.n_tiles = (prm.Sk + TILE - 1) / TILE;
+    FusedParams fp;
+    fp.dq_acc = acc;
+    fp.qscale = qscale;
+    bwd_fused_kernel<D, CAUSAL, F16><<<prm.n_tiles * B * prm.Hkv, FUSED_THREADS, FusedSmem<D>::BYTES, stream>>>(m.q128, m.k128, m.v128, m.do128, prm, fp);
+    if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_fused_kernel launch");
+
+    const long long n_vec = n_rows * prm.d / 8;
+    long long cb = (n_vec + 255) / 256;
+    if (cb > NUM_SMS * 32) cb = NUM_SMS * 32;
+    bwd_dq_convert_kernel<F16><<<static_cast<int>(cb), 256, 0, stream>>>(acc, qscale, prm.dq, n_vec, static_cast<long long>(prm.Sq) * prm.d / 8, prm.scale);
+    if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_dq_convert_kernel launch");
+    return VT_ATTN_OK;
+}
+
 }  // namespace vt
 
 extern "C" size_t vt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int Sq, int Sk, int D)
 {
     vt::Shape s{B, Hq, Hkv, Sq, Sk, D};
     if (vt::check_shape(s, 1.0f) != VT_ATTN_OK) return 0;
+    if (vt::fused_wanted(B, Hq, Hkv, Sq, Sk, D)) return vt::fused_plan(B, Hq, Hkv, Sq, D).total;
     const size_t n = static_cast<size_t>(B) * Hq * Sq * sizeof(float);
     return (n + 255) & ~static_cast<size_t>(255);
+}
+
+extern "C" int vt_attn_bwd_kernel_kind(int B, int Hq, int Hkv, int Sq, int Sk, int D)
+{
+    vt::Shape s{B, Hq, Hkv, Sq, Sk, D};
+    int rc = vt::check_shape(s, 1.0f);
+    if (rc != VT_ATTN_OK) return rc;
+    return vt::fused_wanted(B, Hq, Hkv, Sq, Sk, D) ? 1 : 0;
 }
 
 // Shared by vt_attn_bwd (bfloat16 tensors) and vt_attn_bwd_f16 (IEEE half tensors).
@@ -899,7 +1025,12 @@ static int bwd_entry(bool f16, const void *q, const void *k, const void *v, cons
     if (!ptr_ok(q) || !ptr_ok(k) || !ptr_ok(v) || !ptr_ok(o) || !ptr_ok(d_o) || !ptr_ok(lse, 4) || !ptr_ok(dq) ||
         !ptr_ok(dk) || !ptr_ok(dv) || !ptr_ok(workspace))
         return VT_ATTN_ERR_INVALID_ARGUMENT;
-    if (workspace_bytes < vt_attn_bwd_workspace_bytes(B, Hq, Hkv, Sq, Sk, D)) return VT_ATTN_ERR_WORKSPACE_TOO_SMALL;
+    // The five-product path needs its larger workspace; a caller that brings only the Delta scratch (the static-scratch
+    // entry point does) gets the two-kernel path, which needs nothing else.
+    const size_t split_need = align256(static_cast<size_t>(B) * Hq * Sq * sizeof(float));
+    const bool fused = fused_wanted(B, Hq, Hkv, Sq, Sk, D) && workspace_bytes >= fused_plan(B, Hq, Hkv, Sq, D).total &&
+                       ptr_ok(workspace, 256);
+    if (!fused && workspace_bytes < split_need) return VT_ATTN_ERR_WORKSPACE_TOO_SMALL;
     if (causal < 0 || causal > 2) return VT_ATTN_ERR_INVALID_ARGUMENT;
     rc = check_device();
     if (rc != VT_ATTN_OK) return rc;
@@ -940,6 +1071,12 @@ static int bwd_entry(bool f16, const void *q, const void *k, const void *v, cons
     const __nv_bfloat16 *o_ = static_cast<const __nv_bfloat16 *>(o);
     const __nv_bfloat16 *do_ = static_cast<const __nv_bfloat16 *>(d_o);
     float *delta = static_cast<float *>(workspace);
+    if (fused) {
+        const __nv_bfloat16 *k_ = static_cast<const __nv_bfloat16 *>(k), *v_ = static_cast<const __nv_bfloat16 *>(v);
+        uint8_t *ws = static_cast<uint8_t *>(workspace);
+        if (f16) return causal ? launch_bwd_fused<true, true>(m, prm, o_, do_, k_, v_, ws, B, st) : launch_bwd_fused<false, true>(m, prm, o_, do_, k_, v_, ws, B, st);
+        return causal ? launch_bwd_fused<true, false>(m, prm, o_, do_, k_, v_, ws, B, st) : launch_bwd_fused<false, false>(m, prm, o_, do_, k_, v_, ws, B, st);
+    }
     if (f16) {
         if (Dp == 64)
             return causal ? launch_bwd<64, true, false, true>(m, prm, o_, do_, delta, B, st) : launch_bwd<64, false, false, true>(m, prm, o_, do_, delta, B, st);

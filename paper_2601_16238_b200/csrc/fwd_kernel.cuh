@@ -66,6 +66,10 @@ struct FwdParams {
     long long n_rows;      // B * Hq * Sq (packed batches: total_q * Hq, row = token * Hq + head)
     int hp_tokens;         // PACKED + HPACK: tokens per Q box (the longest sequence's queries)
     int head_group;        // causal kernels: heads per scheduling group (see causal_work_item); 0 or 1: one head after the other
+    // ROPE only: rotary tables [positions, D / 2] (fp32) and the position of query 0 (query i sits at rope_pos0 + i)
+    const float *rope_cos = nullptr;
+    const float *rope_sin = nullptr;
+    int rope_pos0 = 0;
     Guard guard;
 };
 
@@ -76,7 +80,12 @@ struct FwdParams {
 // share the KV head, row = head_in_group * Sq + query, so K / V are walked once for the whole group (decoding shapes).
 // With PACKED the Q box is [tokens][heads], so the row is query * G + head_in_group, and the rows past the sequence's
 // own queries belong to the next sequence (computed, never stored).
-template <int D, bool CAUSAL, bool PACKED, bool SPLIT = false, bool HPACK = false, bool F16 = false>
+// ROPE (batched layout, D = 64 or 128 and equal to the tensors' head dimension): Q arrives unrotated; once the tile is in
+// shared memory every softmax thread turns its own query row by its position's angles ("rotate-half": element i pairs
+// with element i + D / 2), writes it back in the tensors' 16-bit type and only then lets the first product start.  K
+// must come already rotated: a key tile is walked by every query tile of its head, rotating it here would repeat that
+// work once per query tile.
+template <int D, bool CAUSAL, bool PACKED, bool SPLIT = false, bool HPACK = false, bool F16 = false, bool ROPE = false>
 __global__ void __launch_bounds__(FWD_THREADS, 2)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
                 const __grid_constant__ CUtensorMap tm_v, const FwdParams p)
@@ -106,8 +115,10 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     uint64_t *k_empty = bars + 7 + SL;       // [SL]
     uint64_t *v_full = bars + 7 + 2 * SL;    // [SL]
     uint64_t *v_empty = bars + 7 + 3 * SL;   // [SL]
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 7 + 4 * SL);
+    uint64_t *q_rot = bars + 7 + 4 * SL;     // ROPE: 128 arrivals, the query rows have been rotated in place
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 8 + 4 * SL);
     volatile uint32_t *abort_flag = tmem_slot + 1;
+    static_assert(!ROPE || (!PACKED && !SPLIT && !HPACK && (D == 64 || D == 128)), "rotary queries: batched layout, D = 64 or 128");
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -162,6 +173,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         mbar_init(q_full, 1);
         mbar_init(o_final, 1);
         mbar_init(pv_done, 1);
+        if (ROPE) mbar_init(q_rot, 128);
         for (int s = 0; s < 2; ++s) {
             mbar_init(&s_full[s], 1);
             mbar_init(&p_ready[s], 128);
@@ -232,7 +244,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
             const uint32_t IDESC_PV = make_idesc(128, ((p.d + 15) >> 4) * 16, fmt16<F16>(), fmt16<F16>(), 0, 1);
             const uint32_t tmem_u = __shfl_sync(0xFFFFFFFFu, tmem_base, 0);    // provably warp-uniform copy
             const uint64_t dQ0 = smem_desc_sw128(smem_u32(sQ), 16, 1024);
-            bool ok = mbar_wait(q_full, 0, abort_flag, p.guard, status_word(FWD_KERNEL_ID, ROLE_MMA, 0xFFFF));
+            bool ok = mbar_wait(ROPE ? q_rot : q_full, 0, abort_flag, p.guard, status_word(FWD_KERNEL_ID, ROLE_MMA, 0xFFFF));
             if (n_t == 0) ok = false;                     // no keys: nothing to issue (Q was still waited for, so no copy is in flight at exit)
             // S_t = Q K_t^T into S buffer t & 1
             auto issue_qk = [&](int t) -> bool {
@@ -291,7 +303,41 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         float m_used = -INFINITY;                  // maximum (raw scores) the accumulators are scaled by
         float l = 0.0f;
         bool ok = true;
-        for (int t = 0; t < n_t; ++t) {
+        if (ROPE) {
+            // this thread's query row, in place: chunk c (8 elements) of the first half pairs with chunk c of the second
+            // half; in the 128-byte-swizzled tile the 16-byte chunk j of row r sits at chunk j ^ (r & 7) of that row
+            ok = mbar_wait(q_full, 0, abort_flag, p.guard, status_word(FWD_KERNEL_ID, ROLE_SOFTMAX, 0xFFFF));
+            if (ok && q0 + r < Sq) {
+                const size_t pos = static_cast<size_t>(p.rope_pos0 + q0 + r);
+                const float4 *ct = reinterpret_cast<const float4 *>(p.rope_cos + pos * (D / 2));
+                const float4 *st = reinterpret_cast<const float4 *>(p.rope_sin + pos * (D / 2));
+                uint8_t *rowp = sQ + r * 128;
+#pragma unroll
+                for (int ch = 0; ch < D / 16; ++ch) {
+                    uint4 *pa = reinterpret_cast<uint4 *>(rowp + ((ch ^ (r & 7)) << 4));
+                    uint4 *pb = (D == 128) ? reinterpret_cast<uint4 *>(rowp + QBOX_BYTES + ((ch ^ (r & 7)) << 4))
+                                           : reinterpret_cast<uint4 *>(rowp + (((ch + 4) ^ (r & 7)) << 4));
+                    const uint4 a = *pa, bq = *pb;
+                    const float4 c0 = ct[2 * ch], c1 = ct[2 * ch + 1], s0 = st[2 * ch], s1 = st[2 * ch + 1];
+                    const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+                    const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+                    const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {bq.x, bq.y, bq.z, bq.w};
+                    uint32_t ya[4], yb[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const float2 fa = unpack16<F16>(aw[e]), fb = unpack16<F16>(bw[e]);
+                        ya[e] = pack16<F16>(fa.x * cs[2 * e] - fb.x * sn[2 * e], fa.y * cs[2 * e + 1] - fb.y * sn[2 * e + 1]);
+                        yb[e] = pack16<F16>(fb.x * cs[2 * e] + fa.x * sn[2 * e], fb.y * cs[2 * e + 1] + fa.y * sn[2 * e + 1]);
+                    }
+                    *pa = make_uint4(ya[0], ya[1], ya[2], ya[3]);
+                    *pb = make_uint4(yb[0], yb[1], yb[2], yb[3]);
+                }
+            }
+            fence_proxy_async_smem();              // the products read the tile through the async proxy
+            mbar_arrive(q_rot);
+        }
+        const int n_loop = (ROPE && !ok) ? 0 : n_t;         // (a wait gave up while the queries were being rotated)
+        for (int t = 0; t < n_loop; ++t) {
             const uint32_t tS = tmem_base + lane_addr + (t & 1) * BN;
             ok = mbar_wait(&s_full[t & 1], (t >> 1) & 1, abort_flag, p.guard, status_word(FWD_KERNEL_ID, ROLE_SOFTMAX, t));
             if (!ok) break;
@@ -435,7 +481,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
     }
 }
 
-template <int D, bool CAUSAL, bool PACKED, bool SPLIT = false, bool HPACK = false, bool F16 = false>
+template <int D, bool CAUSAL, bool PACKED, bool SPLIT = false, bool HPACK = false, bool F16 = false, bool ROPE = false>
 static int launch_fwd(const CUtensorMap &tq, const CUtensorMap &tk, const CUtensorMap &tv, const FwdParams &prm,
                       int n_blocks, cudaStream_t stream)
 {
@@ -444,11 +490,11 @@ static int launch_fwd(const CUtensorMap &tq, const CUtensorMap &tk, const CUtens
     int dev = 0;
     cudaGetDevice(&dev);
     if (!configured[dev & 63].load(std::memory_order_acquire)) {
-        cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel<D, CAUSAL, PACKED, SPLIT, HPACK, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES);
+        cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel<D, CAUSAL, PACKED, SPLIT, HPACK, F16, ROPE>, cudaFuncAttributeMaxDynamicSharedMemorySize, L::BYTES);
         if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(fwd)");
         configured[dev & 63].store(true, std::memory_order_release);
     }
-    attn_fwd_kernel<D, CAUSAL, PACKED, SPLIT, HPACK, F16><<<n_blocks, FWD_THREADS, L::BYTES, stream>>>(tq, tk, tv, prm);
+    attn_fwd_kernel<D, CAUSAL, PACKED, SPLIT, HPACK, F16, ROPE><<<n_blocks, FWD_THREADS, L::BYTES, stream>>>(tq, tk, tv, prm);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "attn_fwd_kernel launch");
     return VT_ATTN_OK;

@@ -252,18 +252,51 @@ def zigzag_unshard(shards):
     return torch.cat(chunks, dim=2)
 
 
-def _exchange(tensors, nxt, prv, group):
-    """Start sending ``tensors`` to the next rank and receiving their counterparts from the previous one."""
+class _Transfer:
+    """A started exchange.  ``wait()`` orders the caller's later work (on the current stream) behind its completion."""
+
+    def __init__(self, reqs, event=None):
+        self.reqs, self.event = reqs, event
+
+    def wait(self):
+        if self.event is not None:
+            import torch
+            torch.cuda.current_stream().wait_event(self.event)
+        else:
+            for r in self.reqs:
+                r.wait()
+
+
+def _exchange(tensors, nxt, prv, group, comm_stream=None, after_current=True):
+    """Start sending ``tensors`` to the next rank and receiving their counterparts from the previous one.
+
+    ``comm_stream`` (a ``torch.cuda.Stream``, GPU runs only): the point-to-point operations are enqueued there instead of
+    on the current stream, so a step's exchange does not queue behind the attention kernels enqueued before it;
+    ``after_current`` says whether the tensors to send were produced by work on the current stream that the exchange has
+    to wait for (False for blocks that arrived through an earlier exchange on ``comm_stream``).  Returns (transfer, list
+    of receive buffers); the buffers may be read on the current stream after ``transfer.wait()``."""
     import torch
     import torch.distributed as dist
     recv = [torch.empty_like(t) for t in tensors]
     ops = [dist.P2POp(dist.isend, t, nxt, group) for t in tensors] + [dist.P2POp(dist.irecv, t, prv, group) for t in recv]
-    return dist.batch_isend_irecv(ops), recv
+    if comm_stream is None:
+        return _Transfer(dist.batch_isend_irecv(ops)), recv
+    if after_current:
+        comm_stream.wait_stream(torch.cuda.current_stream())
+    for t in list(tensors) + recv:
+        t.record_stream(comm_stream)                 # the allocator must not hand their memory out while the exchange runs
+    with torch.cuda.stream(comm_stream):
+        for r in dist.batch_isend_irecv(ops):
+            r.wait()                                 # orders comm_stream (not the host) behind the library's own stream
+        event = torch.cuda.Event()
+        event.record(comm_stream)
+    return _Transfer([], event), recv
 
 
-def ring_attention_fwd_zigzag(q2, k2, v2, scale: float, group=None, attend=None, merge_factory=None):
+def ring_attention_fwd_zigzag(q2, k2, v2, scale: float, group=None, attend=None, merge_factory=None, comm_stream=None):
     """Causal forward attention in the zig-zag layout.  q2 [2, B, Hq, S_chunk, D], k2 / v2 [2, B, Hkv, S_chunk, D]: this
-    rank's two chunks.  Returns (O2 [2, B, Hq, S_chunk, D], LSE2 [2, B, Hq, S_chunk]).  Collective over ``group``."""
+    rank's two chunks.  Returns (O2 [2, B, Hq, S_chunk, D], LSE2 [2, B, Hq, S_chunk]).  Collective over ``group``.
+    ``comm_stream``: see ``_exchange`` (GPU runs: the K/V blocks travel on a stream of their own)."""
     import torch
     import torch.distributed as dist
     world = dist.get_world_size(group) if dist.is_initialized() else 1
@@ -274,20 +307,19 @@ def ring_attention_fwd_zigzag(q2, k2, v2, scale: float, group=None, attend=None,
     nxt, prv = peer((rank + 1) % world), peer((rank - 1) % world)
     cur_k, cur_v = k2, v2
     for step in range(world):
-        reqs, recv = [], None
+        transfer, recv = None, None
         if step + 1 < world:
-            reqs, recv = _exchange([cur_k, cur_v], nxt, prv, group)
+            transfer, recv = _exchange([cur_k, cur_v], nxt, prv, group, comm_stream, after_current=(step == 0))
         for qi, ki, mode in zigzag_blocks(rank, kv_owner(rank, step, world)):
             merges[qi].add(*attend(q2[qi], cur_k[ki], cur_v[ki], mode, scale))
-        for r in reqs:
-            r.wait()
-        if recv is not None:
+        if transfer is not None:
+            transfer.wait()
             cur_k, cur_v = recv
     (o0, l0), (o1, l1) = merges[0].result(), merges[1].result()
     return torch.stack([torch.as_tensor(o0), torch.as_tensor(o1)]), torch.stack([torch.as_tensor(l0), torch.as_tensor(l1)])
 
 
-def ring_attention_bwd_zigzag(q2, k2, v2, o2, do2, lse2, scale: float, group=None, attend_bwd=None, sum_factory=None):
+def ring_attention_bwd_zigzag(q2, k2, v2, o2, do2, lse2, scale: float, group=None, attend_bwd=None, sum_factory=None, comm_stream=None):
     """Causal backward in the zig-zag layout: (dQ2, dK2, dV2) stacked like the inputs, given the forward's (o2, lse2)."""
     import torch
     import torch.distributed as dist
@@ -302,27 +334,37 @@ def ring_attention_bwd_zigzag(q2, k2, v2, o2, do2, lse2, scale: float, group=Non
     dv = [sum_factory(v2[i]) for i in range(2)]
     cur_k, cur_v = k2, v2
     for step in range(world):
-        reqs, recv = [], None
+        transfer, recv = None, None
         if step + 1 < world:
-            reqs, recv = _exchange([cur_k, cur_v], nxt, prv, group)
+            transfer, recv = _exchange([cur_k, cur_v], nxt, prv, group, comm_stream, after_current=(step == 0))
         for qi, ki, mode in zigzag_blocks(rank, kv_owner(rank, step, world)):
             dq_p, dk_p, dv_p = attend_bwd(q2[qi], cur_k[ki], cur_v[ki], o2[qi], do2[qi], lse2[qi], mode, scale)
             dq[qi].add(dq_p)
             dk[ki].add(dk_p)
             dv[ki].add(dv_p)
-        for r in reqs:
-            r.wait()
+        if transfer is not None:
+            transfer.wait()
         if world > 1:
-            # hand the running dK / dV of the held chunks on (after the last step they are back at their owner)
+            # hand the running dK / dV of the held chunks on (after the last step they are back at their owner); they
+            # were just updated on the current stream, so this exchange has to wait for it
             accs = [dk[0].acc, dk[1].acc, dv[0].acc, dv[1].acc]
-            reqs2, got = _exchange(accs, nxt, prv, group)
-            for r in reqs2:
-                r.wait()
+            transfer2, got = _exchange(accs, nxt, prv, group, comm_stream, after_current=True)
+            transfer2.wait()
             dk[0].acc, dk[1].acc, dv[0].acc, dv[1].acc = got
         if recv is not None:
             cur_k, cur_v = recv
     stack = lambda sums: torch.stack([torch.as_tensor(s.result()) for s in sums])      # noqa: E731
     return stack(dq), stack(dk), stack(dv)
+
+
+def ring_attention_zigzag_fwd_bwd(q2, k2, v2, do2, scale: float, group=None, comm_stream=None, attend=None, merge_factory=None,
+                                  attend_bwd=None, sum_factory=None):
+    """One training step's attention in the zig-zag layout: the causal forward, then the backward for the upstream
+    gradient do2.  Returns (O2, LSE2, dQ2, dK2, dV2).  With one rank (or no process group) nothing is exchanged and the
+    three blocks of the rank's own shard are all there is.  This is what the benchmark workload ``ring_causal_64k`` times."""
+    o2, lse2 = ring_attention_fwd_zigzag(q2, k2, v2, scale, group, attend, merge_factory, comm_stream)
+    dq2, dk2, dv2 = ring_attention_bwd_zigzag(q2, k2, v2, o2, do2, lse2, scale, group, attend_bwd, sum_factory, comm_stream)
+    return o2, lse2, dq2, dk2, dv2
 
 
 def ring_attention_zigzag_local(q2s, k2s, v2s, scale: float, do2s=None, attend=None, merge_factory=None, attend_bwd=None, sum_factory=None):

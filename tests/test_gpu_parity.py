@@ -74,7 +74,16 @@ def test_sdpa_sweep_full_size_whole_tensors(vt, S, causal):
     o, lse = host(o), host(lse)
     o_ref, lse_ref = orc.attn_fwd(q, k, v, cfg.causal, cfg.scale)
     assert o.shape == o_ref.shape == (cfg.B, cfg.Hq, S, cfg.D)
-    assert np.abs(o_ref).max() < 4.0, "bf16 rounding of an output in [4, 8) alone would exceed the O tolerance"
+    # Under the causal mask the first rows of a head reproduce single V rows, and a few of the 8 million N(0,1) values of V
+    # exceed 4 in magnitude: a bf16 output in [4, 8) is spaced 2^-5 apart, so half a spacing (1.6e-2) is the closest any
+    # bf16 result can be guaranteed to come.  Those elements (a handful per tensor, counted below) are held to one bf16
+    # rounding of the exact value, 2^-8 |O|; every other element to the strict 1e-2.
+    big = np.abs(o_ref) >= 4.0
+    assert big.sum() <= 1e-6 * o_ref.size
+    if big.any():
+        assert causal, "only rows that see very few keys can reach |O| >= 4"
+        assert (np.abs(o[big] - o_ref[big]) <= 2.0 ** -8 * np.abs(o_ref[big])).all()
+        o = np.where(big, o_ref, o)          # checked above; the strict gate below covers all the others
     check_fwd(o, lse, o_ref, lse_ref, cfg.name)
 
 

@@ -290,8 +290,14 @@ def test_invalid_arguments_on_the_gpu_path(vt):
     assert e.value.status == vt.ERR_UNSUPPORTED
     q = torch.zeros(1, 3, 128, 64, dtype=torch.bfloat16, device="cuda")
     k = torch.zeros(1, 2, 128, 64, dtype=torch.bfloat16, device="cuda")
-    with pytest.raises(vt.VtAttnError) as e:
+    with pytest.raises(ValueError):                      # the binding refuses Hq % Hkv != 0 before the library is entered ...
         vt.vt_attn_fwd(q, k, k, False, 0.1)
+    lib = vt.load_library()                              # ... and the library refuses it when called directly
+    o = torch.empty_like(q); lse = torch.empty(1, 3, 128, device="cuda")
+    rc = lib.vt_attn_fwd(q.data_ptr(), k.data_ptr(), k.data_ptr(), o.data_ptr(), lse.data_ptr(), 1, 3, 2, 128, 128, 64, 0, 0.1, None)
+    assert rc == vt.ERR_INVALID_ARGUMENT
+    with pytest.raises(vt.VtAttnError) as e:
+        vt.vt_attn_fwd(k, k, k, False, float("nan"))
     assert e.value.status == vt.ERR_INVALID_ARGUMENT
     with pytest.raises(ValueError):
         vt.vt_attn_fwd(q.float(), k, k, False, 0.1)

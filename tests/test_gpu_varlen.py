@@ -82,9 +82,12 @@ def test_packed_argument_checks(vt):
     import torch
     q = torch.zeros(10, 3, 64, dtype=torch.bfloat16, device="cuda"); k = torch.zeros(10, 2, 64, dtype=torch.bfloat16, device="cuda")
     cu = torch.tensor([0, 10], dtype=torch.int32, device="cuda")
-    with pytest.raises(vt.VtAttnError) as e:
-        vt.vt_attn_fwd_varlen(q, k, k, cu, cu, 10, 10, False, 0.1)          # Hq % Hkv != 0
-    assert e.value.status == vt.ERR_INVALID_ARGUMENT
+    with pytest.raises(ValueError):
+        vt.vt_attn_fwd_varlen(q, k, k, cu, cu, 10, 10, False, 0.1)          # Hq % Hkv != 0: refused by the binding ...
+    o = torch.empty_like(q); lse = torch.empty(3, 10, device="cuda")
+    rc = vt.load_library().vt_attn_fwd_varlen(q.data_ptr(), k.data_ptr(), k.data_ptr(), o.data_ptr(), lse.data_ptr(), cu.data_ptr(),
+                                              cu.data_ptr(), 1, 3, 2, 10, 10, 10, 10, 64, 0, 0.1, None)
+    assert rc == vt.ERR_INVALID_ARGUMENT                                    # ... and by the library when called directly
     q = torch.zeros(10, 2, 64, dtype=torch.bfloat16, device="cuda")
     with pytest.raises(vt.VtAttnError) as e:
         vt.vt_attn_fwd_varlen(q, k, k, cu, cu, 11, 10, False, 0.1)          # max_sq > total_q

@@ -232,3 +232,58 @@ def test_zigzag_ring_of_gloo_ranks_forward_and_backward(world):
         assert p.exitcode == 0
     assert [r[0] for r in results] == list(range(world))
     assert all(ef < 1e-12 and eb < 1e-12 for _, ef, eb in results)
+
+
+# ------------------------------------------------------------------------------------------------ the benchmark's ring workload
+def _worker_bench_ring(rank, world, port, out):
+    """The benchmark's own step function and input generator (bench.ring_step / bench.ring_shard_bits) on gloo ranks,
+    with the oracle-built stand-ins for the kernels."""
+    os.environ.update(RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(world), MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    import torch
+    import torch.distributed as dist
+    import bench
+    from oracle import attn_oracle as orc
+    from paper_2601_16238_b200.ring import zigzag_shard, zigzag_unshard
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    w = {"B": 1, "Hq": 4, "Hkv": 2, "S": 96, "D": 8, "pieces": 8, "index": 77}
+    scale = 0.3
+    wide = lambda bits: torch.from_numpy(orc.bf16_bits_to_f64(bits))       # noqa: E731
+    mine = [wide(x) for x in bench.ring_shard_bits(w, rank, world)]
+    # every world size must see the same sequence: rebuild it from all ranks' shards and from a one-rank run
+    full = [zigzag_unshard([wide(bench.ring_shard_bits(w, r, world)[t]) for r in range(world)]) for t in range(4)]
+    alone = [zigzag_unshard([wide(bench.ring_shard_bits(w, 0, 1)[t])]) for t in range(4)]
+    same = all(torch.equal(a, b) for a, b in zip(full, alone))
+
+    def attend(q_, k_, v_, mode, scale_):
+        return orc.attn_fwd(q_.numpy(), k_.numpy(), v_.numpy(), mode, scale_)
+
+    o2, lse2, dq2, dk2, dv2 = bench.ring_step(*mine, scale, attend=attend, merge_factory=lambda q_: _OracleMerge(q_.numpy()),
+                                              attend_bwd=_block_grads, sum_factory=_OracleSum)
+    q, k, v, d_o = (x.numpy() for x in full)
+    o_ref, lse_ref = orc.attn_fwd(q, k, v, True, scale)
+    refs = orc.attn_bwd(q, k, v, d_o, True, scale)
+    sh = lambda x: zigzag_shard(torch.from_numpy(x), rank, world).numpy()      # noqa: E731
+    err = max(float(np.abs(np.asarray(o2) - sh(o_ref)).max()), float(np.abs(np.asarray(lse2) - sh(lse_ref[..., None])[..., 0]).max()),
+              *(float(np.abs(np.asarray(g) - sh(r)).max()) for g, r in zip((dq2, dk2, dv2), refs)))
+    out.put((rank, same, err))
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world", [2, 4])
+def test_benchmark_ring_workload_on_gloo_ranks(world):
+    import torch.multiprocessing as mp
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_worker_bench_ring, args=(r, world, port, out)) for r in range(world)]
+    for p in procs:
+        p.start()
+    results = sorted(out.get(timeout=180) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert [r[0] for r in results] == list(range(world))
+    assert all(same for _, same, _ in results), "every world size must be given the same sequence"
+    assert all(err < 1e-12 for _, _, err in results)
