@@ -37,11 +37,11 @@
  *     *_host entry points serialise their enqueueing inside the library (one call at a
  *     time forks onto the library's two streams and joins back), and two such calls
  *     that are in flight together on one device must not share a staging area.
- *   - Supported: D a multiple of 8 in [8, 128]; in the forward entry points that take
- *     [B, H, S, D] tensors (vt_attn_fwd, vt_attn_fwd_f16, vt_attn_fwd_splitkv) and the merge
- *     entry points up to 256.  The kernels are built for 64, 128 and (forward) 256 columns;
- *     another D runs in the next larger one at that one's cost, its rows are still D
- *     elements long in memory.  B, Hq, Hkv, Sq, Sk >= 1; Hq % Hkv == 0;
+ *   - Supported: D a multiple of 8 in [8, 128]; in the entry points that take
+ *     [B, H, S, D] tensors (vt_attn_fwd, vt_attn_bwd, their _f16 twins, vt_attn_fwd_splitkv)
+ *     and the merge entry points up to 256.  The kernels are built for 64, 128 and 256
+ *     columns; another D runs in the next larger one at that one's cost, its rows are still
+ *     D elements long in memory.  B, Hq, Hkv, Sq, Sk >= 1; Hq % Hkv == 0;
  *     B * Hq and B * Hkv at most 2^31 - 1; Sq, Sk at most 2^24; scale finite, > 0.
  */
 #ifndef VT_ATTN_H_
@@ -57,7 +57,7 @@ extern "C" {
 
 #define VT_ATTN_OK 0
 #define VT_ATTN_ERR_INVALID_ARGUMENT (-1)    /* null/misaligned pointer, bad shape or scale */
-#define VT_ATTN_ERR_UNSUPPORTED (-2)         /* head dim not a multiple of 8 in [8,128] ([8,256] forward); device is not sm_100 */
+#define VT_ATTN_ERR_UNSUPPORTED (-2)         /* head dim not a multiple of 8 in [8,256] ([8,128] in the packed and host-buffer entry points); device is not sm_100 */
 #define VT_ATTN_ERR_WORKSPACE_TOO_SMALL (-3) /* workspace_bytes below vt_attn_bwd_workspace_bytes */
 #define VT_ATTN_ERR_CUDA (-4)                /* a CUDA runtime / driver call failed */
 #define VT_ATTN_ERR_DEVICE_TIMEOUT (-5)      /* reported by vt_attn_device_status only */
@@ -127,7 +127,10 @@ size_t vt_attn_bwd_workspace_bytes(int B, int Hq, int Hkv, int Sq, int Sk, int D
  *      in 32-bit fixed point, scaled per (batch, head) from bounds on dO, K and V, so the sum
  *      does not depend on the order in which the blocks add and dQ is the same bits on every
  *      run; a last pass rounds it to the tensors' type.  Six kernels and one memset per call.
- * The library itself always answers 0: on the B200 the reductions of 1 cost more than the two
+ *   2  D above 128 (up to 256): Delta, a dK / dV kernel that keeps 128 keys stationary and
+ *      walks the queries 64 at a time, once per half of the output columns, and a dQ kernel
+ *      that keeps 128 queries stationary and walks the keys 64 at a time.
+ * For D <= 128 the library itself always answers 0: on the B200 the reductions of 1 cost more than the two
  * products they save.  The environment variable VT_ATTN_BWD_PATH=fused (read at every call)
  * selects 1 wherever it is built, for measurements and tests; =split or unset selects 0.  A
  * call whose workspace only holds Delta (vt_attn_bwd_static_scratch does this) takes 0 too.

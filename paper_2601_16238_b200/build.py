@@ -17,7 +17,7 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libvtattn.so")
 BUILD_DIR = os.path.join(HERE, "build")
 
-SOURCES = ["common.cu", "fwd.cu", "fwd_rope.cu", "fwd_split.cu", "merge.cu", "bwd.cu", "host_api.cu", "selftest.cu", "suite.cu"]
+SOURCES = ["common.cu", "fwd.cu", "fwd_rope.cu", "fwd_split.cu", "merge.cu", "bwd.cu", "bwd_wide.cu", "host_api.cu", "selftest.cu", "suite.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math", "-I", INCLUDE]
 

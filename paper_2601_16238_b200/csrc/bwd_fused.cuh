@@ -462,7 +462,6 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
             const int q0 = (qt_start + qi) * TILE;
             int *dst = fp.dq_acc + ((static_cast<size_t>(b) * p.Hq + hq) * p.Sq + q0) * p.d + dcol;
             const int n_valid = min(TILE, Sq - q0);                // query rows of this tile that exist
-#ifndef VT_FUSED_DBG_NO_RED
             if (dcol < p.d) {
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
@@ -475,9 +474,6 @@ bwd_fused_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant
                     }
                 }
             }
-#else
-            if (v[0][0] == 0x12345678u && v[3][31] == 0x9abcdef0u) dst[0] = n_valid + static_cast<int>(qs);     // keeps the loads alive
-#endif
             if (++qi == n_qi) {
                 qi = 0;
                 ++hq;

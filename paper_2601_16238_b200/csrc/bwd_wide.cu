@@ -1,0 +1,713 @@
+// Backward fused attention for head dimensions in (128, 256] (batched layout).
+//
+// The 128-column kernels of bwd.cu keep two 128-row operand tiles stationary in shared memory and four 128-column
+// accumulators in tensor memory; at 256 columns neither fits.  Here the stationary side stays 128 rows (at 256 columns:
+// 64 KB per tile) and the streamed side is cut to 64 rows, so every score tile is 128 x 64:
+//
+//   bwd_dkdv_wide_kernel : one block per (batch, KV head, 128-key tile, column half).  K and V (all 256 columns) stay in
+//       shared memory; the query heads of the group are walked 64 queries at a time (Q in two slots, dO in one).
+//       S^T = K Q^T and dP^T = V dO^T contract over all columns; dV and dK are accumulated for ONE half of the
+//       columns per block (two accumulators of 128 columns next to S^T and dP^T in tensor memory), so the grid's
+//       second dimension runs the walk twice - the price of 512 tensor-memory columns.
+//   bwd_dq_wide_kernel   : one block per (batch, query head, 128-query tile).  Q and dO stay in shared memory, K (two
+//       slots) and V (one slot) stream by in tiles of 64 keys; dQ (256 columns) is accumulated in tensor memory.
+//
+// Same roles as in bwd.cu (warp 0 / 2 TMA producers, warp 1 MMA issuer, warp 3 row-vector producer) with ONE compute
+// warpgroup (warps 4..7: a 128 x 64 tile is what one warpgroup of the 128-column kernels handles).  Every output tile
+// has one owner block and every sum a fixed order, as there.  Delta comes from bwd_delta_kernel.
+#include <mutex>
+
+#include "bwd_common.cuh"
+
+namespace vt {
+
+constexpr int WIDE_D = 256;                          // columns the kernels are built for (the real head dimension d <= 256)
+constexpr int WIDE_THREADS = 256;
+constexpr int WIDE_N = 64;                           // rows of a streamed tile = columns of a score tile
+constexpr int WIDE_BOXES = WIDE_D / BOX_COLS;        // 4 boxes of 64 columns per row
+constexpr int BOX128_BYTES = TILE * BOX_COLS * 2;    // 16 KB: one box of a 128-row tile
+constexpr int BOX64_BYTES = WIDE_N * BOX_COLS * 2;   // 8 KB: one box of a 64-row tile
+constexpr int TILE128_BYTES = WIDE_BOXES * BOX128_BYTES;   // 64 KB
+constexpr int TILE64_BYTES = WIDE_BOXES * BOX64_BYTES;     // 32 KB
+constexpr uint32_t DKDV_WIDE_KERNEL_ID = 6;
+constexpr uint32_t DQ_WIDE_KERNEL_ID = 7;
+
+struct DkdvWideSmem {
+    static constexpr int OFF_K = 0;
+    static constexpr int OFF_V = OFF_K + TILE128_BYTES;
+    static constexpr int OFF_Q = OFF_V + TILE128_BYTES;              // [2]
+    static constexpr int OFF_DO = OFF_Q + 2 * TILE64_BYTES;          // [1]
+    static constexpr int ROW_SLOTS = 2;
+    static constexpr int OFF_ROWS = OFF_DO + TILE64_BYTES;           // [slot][-lse2 64 | -delta 64]
+    static constexpr int OFF_BAR = OFF_ROWS + ROW_SLOTS * 2 * WIDE_N * 4;
+    static constexpr int BYTES = OFF_BAR + 256;                      // no alignment slack: the kernel checks the base address
+    // TMEM columns: S^T [0,64) (P^T, bf16, over its first 32), dP^T [64,128) (dS^T over its first 32), dV half [128,256),
+    // dK half [256,384)
+    static constexpr int TMEM_COLS = 512;
+};
+
+template <bool CAUSAL, bool F16>
+__global__ void __launch_bounds__(WIDE_THREADS, 1)
+bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                     const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, const BwdParams p)
+{
+    using L = DkdvWideSmem;
+    constexpr int RS = L::ROW_SLOTS;
+    extern __shared__ __align__(1024) uint8_t smem_wide[];
+    uint8_t *smem = smem_wide;
+    uint8_t *sK = smem + L::OFF_K;
+    uint8_t *sV = smem + L::OFF_V;
+    uint8_t *sQ = smem + L::OFF_Q;
+    uint8_t *sdO = smem + L::OFF_DO;
+    float *s_rows = reinterpret_cast<float *>(smem + L::OFF_ROWS);
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::OFF_BAR);
+    uint64_t *kv_full = bars + 0;
+    uint64_t *final_bar = bars + 1;
+    uint64_t *s_full = bars + 2;
+    uint64_t *dp_full = bars + 3;
+    uint64_t *p_ready = bars + 4;             // 128 arrivals
+    uint64_t *ds_ready = bars + 5;            // 128 arrivals
+    uint64_t *q_full = bars + 6;              // [2]
+    uint64_t *q_empty = bars + 8;             // [2]
+    uint64_t *do_full = bars + 10;
+    uint64_t *do_empty = bars + 11;
+    uint64_t *rows_full = bars + 12;          // [RS] 32 arrivals
+    uint64_t *rows_empty = bars + 12 + RS;    // [RS] one arrival per compute warp
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 12 + 2 * RS);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    if ((smem_u32(smem_wide) & 1023u) != 0u) {           // the swizzled tiles need this, and there is no room for slack
+        if (threadIdx.x == 0) atomicCAS(p.guard.status, 0u, status_word(DKDV_WIDE_KERNEL_ID, ROLE_LOAD, 0xFFFE));
+        return;
+    }
+
+    const int half = blockIdx.y;                          // which 128 columns of dK / dV this block accumulates
+    const int bh_kv = blockIdx.x / p.n_tiles;
+    const int kt = blockIdx.x % p.n_tiles;
+    const int b = bh_kv / p.Hkv;
+    const int hkv = bh_kv % p.Hkv;
+    const int k0 = kt * TILE;
+    const int Sq = p.Sq, Sk = p.Sk;
+    const int n_qt = (Sq + WIDE_N - 1) / WIDE_N;          // 64-query tiles per head
+    const int off = (CAUSAL && p.bottom_right) ? Sk - Sq : 0;
+    const int qt_start = CAUSAL ? min(max(k0 - off, 0) / WIDE_N, n_qt) : 0;   // first query tile with a query that sees key k0
+    const int n_qi = n_qt - qt_start;
+    const int n_it = n_qi * p.G;
+    const int cols_out = min(TILE, p.d - half * TILE);    // real columns of this half (> 0: d > 128)
+    const int kd = (p.d + 15) >> 4;                       // 16-column contraction steps that hold data
+
+    if (threadIdx.x == 0) {
+        mbar_init(kv_full, 1);
+        mbar_init(final_bar, 1);
+        mbar_init(s_full, 1);
+        mbar_init(dp_full, 1);
+        mbar_init(p_ready, 128);
+        mbar_init(ds_ready, 128);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&q_full[s], 1);
+            mbar_init(&q_empty[s], 1);
+        }
+        mbar_init(do_full, 1);
+        mbar_init(do_empty, 1);
+        for (int s = 0; s < RS; ++s) {
+            mbar_init(&rows_full[s], 32);
+            mbar_init(&rows_empty[s], 4);
+        }
+        *abort_flag = 0u;
+        fence_mbar_init();
+        prefetch_tensormap(&tm_q);
+        prefetch_tensormap(&tm_k);
+        prefetch_tensormap(&tm_v);
+        mbar_arrive_expect_tx(kv_full, 2 * TILE128_BYTES);
+        for (int kb = 0; kb < WIDE_BOXES; ++kb) {
+            tma_load_3d(sK + kb * BOX128_BYTES, &tm_k, kv_full, kb * BOX_COLS, k0, bh_kv);
+            tma_load_3d(sV + kb * BOX128_BYTES, &tm_v, kv_full, kb * BOX_COLS, k0, bh_kv);
+        }
+        if (n_it > 0) {
+            mbar_arrive_expect_tx(&q_full[0], TILE64_BYTES);
+            for (int kb = 0; kb < WIDE_BOXES; ++kb)
+                tma_load_3d(sQ + kb * BOX64_BYTES, &tm_q, &q_full[0], kb * BOX_COLS, qt_start * WIDE_N, b * p.Hq + hkv * p.G);
+        }
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, L::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {                           // Q tiles (K, V and the first one went out before the block-wide sync)
+            for (int it = 1; it < n_it; ++it) {
+                const int sl = it & 1;
+                const int hq = hkv * p.G + it / n_qi;
+                const int q0 = (qt_start + it % n_qi) * WIDE_N;
+                if (!mbar_wait(&q_empty[sl], ((it >> 1) & 1) ^ 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_LOAD, it))) break;
+                mbar_arrive_expect_tx(&q_full[sl], TILE64_BYTES);
+                for (int kb = 0; kb < WIDE_BOXES; ++kb)
+                    tma_load_3d(sQ + sl * TILE64_BYTES + kb * BOX64_BYTES, &tm_q, &q_full[sl], kb * BOX_COLS, q0, b * p.Hq + hq);
+            }
+        }
+    } else if (warp == 2) {
+        if (lane == 0) {                           // dO tiles: one slot, reloaded as soon as dV of the iteration has completed
+            prefetch_tensormap(&tm_do);
+            for (int it = 0; it < n_it; ++it) {
+                const int hq = hkv * p.G + it / n_qi;
+                const int q0 = (qt_start + it % n_qi) * WIDE_N;
+                if (!mbar_wait(do_empty, (it & 1) ^ 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_LOAD, it))) break;
+                mbar_arrive_expect_tx(do_full, TILE64_BYTES);
+                for (int kb = 0; kb < WIDE_BOXES; ++kb)
+                    tma_load_3d(sdO + kb * BOX64_BYTES, &tm_do, do_full, kb * BOX_COLS, q0, b * p.Hq + hq);
+            }
+        }
+    } else if (warp == 3) {
+        // row vectors of the iteration's 64 queries: -LSE (log2 units; -inf past the end, so P = 0) and -Delta
+        for (int it = 0; it < n_it; ++it) {
+            const int sl = it % RS;
+            if (!mbar_wait(&rows_empty[sl], ((it / RS) & 1) ^ 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_LOAD, it))) break;
+            const int hq = hkv * p.G + it / n_qi;
+            const int q0 = (qt_start + it % n_qi) * WIDE_N;
+            const size_t head = (static_cast<size_t>(b) * p.Hq + hq) * p.Sq;
+            float *dst = s_rows + sl * (2 * WIDE_N);
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                const int q = q0 + e * 32 + lane;
+                float nl = -INFINITY, nd = 0.0f;
+                if (q < Sq) {
+                    nl = -p.lse[head + q] * LOG2E;
+                    nd = -p.delta[head + q];
+                }
+                dst[e * 32 + lane] = nl;
+                dst[WIDE_N + e * 32 + lane] = nd;
+            }
+            mbar_arrive(&rows_full[sl]);
+        }
+    } else if (warp == 1) {
+        // MMA issuer.  Per iteration: dV(i), S(i+1), dK(i), dP(i+1) - the order of the 128-column kernel.
+        constexpr uint32_t IDESC_S = make_idesc(128, WIDE_N, fmt16<F16>(), fmt16<F16>(), 0, 0);
+        const uint32_t IDESC_G = make_idesc(128, ((cols_out + 15) >> 4) * 16, fmt16<F16>(), fmt16<F16>(), 0, 1);
+        const uint32_t tmem_u = __shfl_sync(0xFFFFFFFFu, tmem_base, 0);
+        const uint64_t dK0 = smem_desc_sw128(smem_u32(sK), 16, 1024), dV0 = smem_desc_sw128(smem_u32(sV), 16, 1024);
+        // dO and Q as MN-major B operands restricted to this block's column half: boxes 2 * half and 2 * half + 1
+        const uint64_t dDOm = smem_desc_sw128(smem_u32(sdO + half * 2 * BOX64_BYTES), BOX64_BYTES, 1024);
+        bool ok = mbar_wait(kv_full, 0, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, 0xFFFF));
+        auto issue_s = [&](int it) -> bool {       // S^T = K Q^T over all columns
+            const int sl = it & 1;
+            if (!mbar_wait(&q_full[sl], (it >> 1) & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it))) return false;
+            tc_fence_after_sync();
+            if (elect_one()) {
+                const uint64_t dQs = smem_desc_sw128(smem_u32(sQ + sl * TILE64_BYTES), 16, 1024);
+#pragma unroll
+                for (int k = 0; k < WIDE_D / 16; ++k)
+                    if (k < kd)
+                        umma_ss(tmem_u, desc_advance(dK0, (k / 4) * BOX128_BYTES + (k % 4) * 32),
+                                desc_advance(dQs, (k / 4) * BOX64_BYTES + (k % 4) * 32), IDESC_S, k > 0 ? 1u : 0u);
+                umma_commit(s_full);
+            }
+            __syncwarp();
+            return true;
+        };
+        auto issue_dp = [&](int it) -> bool {      // dP^T = V dO^T over all columns
+            if (!mbar_wait(do_full, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it))) return false;
+            tc_fence_after_sync();
+            if (elect_one()) {
+                const uint64_t dDOs = smem_desc_sw128(smem_u32(sdO), 16, 1024);
+#pragma unroll
+                for (int k = 0; k < WIDE_D / 16; ++k)
+                    if (k < kd)
+                        umma_ss(tmem_u + 64, desc_advance(dV0, (k / 4) * BOX128_BYTES + (k % 4) * 32),
+                                desc_advance(dDOs, (k / 4) * BOX64_BYTES + (k % 4) * 32), IDESC_S, k > 0 ? 1u : 0u);
+                umma_commit(dp_full);
+            }
+            __syncwarp();
+            return true;
+        };
+        if (ok && n_it > 0) ok = issue_s(0);
+        if (ok && n_it > 0) ok = issue_dp(0);
+        for (int it = 0; it < n_it && ok; ++it) {
+            const int sl = it & 1;
+            ok = mbar_wait(p_ready, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it));
+            if (!ok) break;
+            tc_fence_after_sync();
+            if (elect_one()) {                     // dV[:, half] += P^T dO[:, half]   (16 query rows per instruction)
+#pragma unroll
+                for (int k = 0; k < WIDE_N / 16; ++k)
+                    umma_ts(tmem_u + 128, tmem_u + k * 8, desc_advance(dDOm, k * 2048), IDESC_G, (it > 0 || k > 0) ? 1u : 0u);
+                umma_commit(do_empty);
+            }
+            __syncwarp();
+            if (it + 1 < n_it) {
+                ok = issue_s(it + 1);              // overwrites P^T(it): ordered behind dV(it)
+                if (!ok) break;
+            }
+            ok = mbar_wait(ds_ready, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it));
+            if (!ok) break;
+            tc_fence_after_sync();
+            if (elect_one()) {                     // dK[:, half] += dS^T Q[:, half]
+                const uint64_t dQm = smem_desc_sw128(smem_u32(sQ + sl * TILE64_BYTES + half * 2 * BOX64_BYTES), BOX64_BYTES, 1024);
+#pragma unroll
+                for (int k = 0; k < WIDE_N / 16; ++k)
+                    umma_ts(tmem_u + 256, tmem_u + 64 + k * 8, desc_advance(dQm, k * 2048), IDESC_G, (it > 0 || k > 0) ? 1u : 0u);
+                umma_commit(&q_empty[sl]);
+                if (it == n_it - 1) umma_commit(final_bar);
+            }
+            __syncwarp();
+            if (it + 1 < n_it) ok = issue_dp(it + 1);     // overwrites dS^T(it): ordered behind dK(it)
+        }
+    } else if (warp >= 4) {
+        // compute: P^T, dS^T (fragment-shaped tensor-memory accesses, see vt_ptx.cuh); epilogue
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;            // key row inside the tile (TMEM lane)
+        const int kv = k0 + r;
+        const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
+        const uint32_t tS = tmem_base + lane_addr;
+        const uint32_t tDP = tmem_base + lane_addr + 64;
+        const float2 c2 = make_float2(p.scale_log2e, p.scale_log2e);
+        const int cq = 2 * (lane & 3);
+        const int kv_row = k0 + quad * 32 + (lane >> 2);
+        bool ok = true;
+        int qi = 0;
+        for (int it = 0; it < n_it; ++it, qi = (qi + 1 == n_qi) ? 0 : qi + 1) {
+            const int q0 = (qt_start + qi) * WIDE_N;
+            const int rsl = it % RS;
+            const float *rows = s_rows + rsl * (2 * WIDE_N);
+            ok = mbar_wait(&rows_full[rsl], (it / RS) & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_SOFTMAX, it));
+            if (!ok) break;
+            ok = mbar_wait(s_full, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_SOFTMAX, it));
+            if (!ok) break;
+            tc_fence_after_sync();
+            const bool diag = CAUSAL && (q0 + off < k0 + TILE - 1);
+            float2 nl[8];
+#pragma unroll
+            for (int g = 0; g < 8; ++g) nl[g] = *reinterpret_cast<const float2 *>(&rows[8 * g + cq]);
+            float2 pr[2][8][2];
+            uint32_t sv[2][32];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) tmem_ld_frag64(tS + (static_cast<uint32_t>(h * 16) << 16), sv[h]);
+            tmem_wait_ld();
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t pp[16];
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+#pragma unroll
+                    for (int rr = 0; rr < 2; ++rr) {
+                        const float2 x = __ffma2_rn(make_float2(__uint_as_float(sv[h][4 * g + 2 * rr]), __uint_as_float(sv[h][4 * g + 2 * rr + 1])),
+                                                    c2, nl[g]);
+                        float2 e = prob_pair(2 * g + rr, x);
+                        if (diag) {
+                            const int kvr = kv_row + 16 * h + 8 * rr;
+                            if (q0 + 8 * g + cq + off < kvr) e.x = 0.0f;
+                            if (q0 + 8 * g + cq + 1 + off < kvr) e.y = 0.0f;
+                        }
+                        pr[h][g][rr] = e;
+                        pp[2 * g + rr] = pack16<F16>(e.x, e.y);
+                    }
+                }
+                tmem_st_frag32(tS + (static_cast<uint32_t>(h * 16) << 16), pp);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(p_ready);
+#pragma unroll
+            for (int g = 0; g < 8; ++g) nl[g] = *reinterpret_cast<const float2 *>(&rows[WIDE_N + 8 * g + cq]);   // now -delta
+            ok = mbar_wait(dp_full, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_SOFTMAX, it));
+            if (!ok) break;
+            tc_fence_after_sync();
+#pragma unroll
+            for (int h = 0; h < 2; ++h) tmem_ld_frag64(tDP + (static_cast<uint32_t>(h * 16) << 16), sv[h]);
+            tmem_wait_ld();
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                uint32_t dd[16];
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+#pragma unroll
+                    for (int rr = 0; rr < 2; ++rr) {
+                        const float2 df = __fadd2_rn(make_float2(__uint_as_float(sv[h][4 * g + 2 * rr]), __uint_as_float(sv[h][4 * g + 2 * rr + 1])), nl[g]);
+                        const float2 ds = __fmul2_rn(pr[h][g][rr], df);
+                        dd[2 * g + rr] = pack16<F16>(ds.x, ds.y);
+                    }
+                }
+                tmem_st_frag32(tDP + (static_cast<uint32_t>(h * 16) << 16), dd);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(ds_ready);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&rows_empty[rsl]);
+        }
+        // epilogue: this block's column half of dV, then of dK
+        const size_t row_off = (static_cast<size_t>(bh_kv) * p.Sk + kv) * p.d + half * TILE;
+        if (n_it == 0) {
+            if (kv < Sk)
+                for (int i = 0; i < cols_out / 8; ++i) {
+                    reinterpret_cast<uint4 *>(p.dv + row_off)[i] = make_uint4(0, 0, 0, 0);
+                    reinterpret_cast<uint4 *>(p.dk + row_off)[i] = make_uint4(0, 0, 0, 0);
+                }
+        } else {
+            if (ok) ok = mbar_wait(final_bar, 0, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_EPILOGUE, 0));
+            if (ok) {
+                tc_fence_after_sync();
+                uint8_t *scratch = sQ + (warp - 4) * STORE_SCRATCH_BYTES;     // every product has completed: the Q slots are free
+                const int row0 = k0 + quad * 32;
+                const size_t stride = static_cast<size_t>(p.d);
+                const int rows_valid = min(32, Sk - row0);
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    __nv_bfloat16 *warp_dst = (t == 0 ? p.dv : p.dk) + row_off - static_cast<size_t>(lane) * stride;
+                    const uint32_t tSrc = tmem_base + lane_addr + 128 + t * 128;
+                    const float mul = (t == 0) ? 1.0f : p.scale;
+#pragma unroll
+                    for (int c = 0; c < TILE / 32; ++c) {
+                        uint32_t v[32];
+                        tmem_ld32(tSrc + c * 32, v);
+                        tmem_wait_ld();
+                        store_rows16<F16>(warp_dst + c * 32, stride, v, mul, rows_valid, scratch, lane, cols_out - c * 32);
+                    }
+                }
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, L::TMEM_COLS);
+    }
+}
+
+// ----------------------------------------------------------------------------------------------
+// dQ, query tile stationary
+// ----------------------------------------------------------------------------------------------
+struct DqWideSmem {
+    static constexpr int OFF_Q = 0;
+    static constexpr int OFF_DO = OFF_Q + TILE128_BYTES;
+    static constexpr int OFF_K = OFF_DO + TILE128_BYTES;             // [2] tiles of 64 keys
+    static constexpr int OFF_V = OFF_K + 2 * TILE64_BYTES;           // [1]
+    static constexpr int OFF_BAR = OFF_V + TILE64_BYTES;
+    static constexpr int BYTES = OFF_BAR + 256;
+    // TMEM columns: S [0,64), dP [64,128) (dS, bf16, over its first 32), dQ [128,384)
+    static constexpr int TMEM_COLS = 512;
+};
+
+template <bool CAUSAL, bool F16>
+__global__ void __launch_bounds__(WIDE_THREADS, 1)
+bwd_dq_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                   const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_do, const BwdParams p)
+{
+    using L = DqWideSmem;
+    extern __shared__ __align__(1024) uint8_t smem_wide[];
+    uint8_t *smem = smem_wide;
+    uint8_t *sQ = smem + L::OFF_Q;
+    uint8_t *sdO = smem + L::OFF_DO;
+    uint8_t *sK = smem + L::OFF_K;
+    uint8_t *sV = smem + L::OFF_V;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::OFF_BAR);
+    uint64_t *qdo_full = bars + 0;
+    uint64_t *final_bar = bars + 1;
+    uint64_t *s_full = bars + 2;
+    uint64_t *dp_full = bars + 3;
+    uint64_t *ds_ready = bars + 4;            // 128 arrivals
+    uint64_t *k_full = bars + 5;              // [2]
+    uint64_t *k_empty = bars + 7;             // [2]
+    uint64_t *v_full = bars + 9;
+    uint64_t *v_empty = bars + 10;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 11);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    if ((smem_u32(smem_wide) & 1023u) != 0u) {
+        if (threadIdx.x == 0) atomicCAS(p.guard.status, 0u, status_word(DQ_WIDE_KERNEL_ID, ROLE_LOAD, 0xFFFE));
+        return;
+    }
+
+    const int bh = blockIdx.x / p.n_tiles;
+    int qt = blockIdx.x % p.n_tiles;
+    if (CAUSAL) qt = p.n_tiles - 1 - qt;                   // long (late) tiles first
+    const int b = bh / p.Hq;
+    const int h = bh % p.Hq;
+    const int bh_kv = b * p.Hkv + h / p.G;
+    const int q0 = qt * TILE;
+    const int Sq = p.Sq, Sk = p.Sk;
+    const int off = (CAUSAL && p.bottom_right) ? Sk - Sq : 0;
+    int n_it = (Sk + WIDE_N - 1) / WIDE_N;                 // steps of 64 keys
+    if (CAUSAL) n_it = (q0 + TILE - 1 + off < 0) ? 0 : min(n_it, (q0 + TILE - 1 + off) / WIDE_N + 1);
+    const int kd = (p.d + 15) >> 4;
+
+    if (threadIdx.x == 0) {
+        mbar_init(qdo_full, 1);
+        mbar_init(final_bar, 1);
+        mbar_init(s_full, 1);
+        mbar_init(dp_full, 1);
+        mbar_init(ds_ready, 128);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&k_full[s], 1);
+            mbar_init(&k_empty[s], 1);
+        }
+        mbar_init(v_full, 1);
+        mbar_init(v_empty, 1);
+        *abort_flag = 0u;
+        fence_mbar_init();
+        prefetch_tensormap(&tm_q);
+        prefetch_tensormap(&tm_do);
+        prefetch_tensormap(&tm_k);
+        mbar_arrive_expect_tx(qdo_full, 2 * TILE128_BYTES);
+        for (int kb = 0; kb < WIDE_BOXES; ++kb) {
+            tma_load_3d(sQ + kb * BOX128_BYTES, &tm_q, qdo_full, kb * BOX_COLS, q0, bh);
+            tma_load_3d(sdO + kb * BOX128_BYTES, &tm_do, qdo_full, kb * BOX_COLS, q0, bh);
+        }
+        if (n_it > 0) {
+            mbar_arrive_expect_tx(&k_full[0], TILE64_BYTES);
+            for (int kb = 0; kb < WIDE_BOXES; ++kb) tma_load_3d(sK + kb * BOX64_BYTES, &tm_k, &k_full[0], kb * BOX_COLS, 0, bh_kv);
+        }
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, L::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {                           // K tiles (Q, dO and the first one went out before the block-wide sync)
+            for (int j = 1; j < n_it; ++j) {
+                const int sl = j & 1;
+                if (!mbar_wait(&k_empty[sl], ((j >> 1) & 1) ^ 1, abort_flag, p.guard, status_word(DQ_WIDE_KERNEL_ID, ROLE_LOAD, j))) break;
+                mbar_arrive_expect_tx(&k_full[sl], TILE64_BYTES);
+                for (int kb = 0; kb < WIDE_BOXES; ++kb)
+                    tma_load_3d(sK + sl * TILE64_BYTES + kb * BOX64_BYTES, &tm_k, &k_full[sl], kb * BOX_COLS, j * WIDE_N, bh_kv);
+            }
+        }
+    } else if (warp == 2) {
+        if (lane == 0) {                           // V tiles: one slot
+            prefetch_tensormap(&tm_v);
+            for (int j = 0; j < n_it; ++j) {
+                if (!mbar_wait(v_empty, (j & 1) ^ 1, abort_flag, p.guard, status_word(DQ_WIDE_KERNEL_ID, ROLE_LOAD, j))) break;
+                mbar_arrive_expect_tx(v_full, TILE64_BYTES);
+                for (int kb = 0; kb < WIDE_BOXES; ++kb) tma_load_3d(sV + kb * BOX64_BYTES, &tm_v, v_full, kb * BOX_COLS, j * WIDE_N, bh_kv);
+            }
+        }
+    } else if (warp == 1) {
+        // MMA issuer.  Per step: dQ(j), S(j+1), dP(j+1).
+        constexpr uint32_t IDESC_S = make_idesc(128, WIDE_N, fmt16<F16>(), fmt16<F16>(), 0, 0);
+        const uint32_t IDESC_G = make_idesc(128, kd * 16, fmt16<F16>(), fmt16<F16>(), 0, 1);     // N = the head dimension, up to 256
+        const uint32_t tmem_u = __shfl_sync(0xFFFFFFFFu, tmem_base, 0);
+        const uint64_t dQ0 = smem_desc_sw128(smem_u32(sQ), 16, 1024), dDO0 = smem_desc_sw128(smem_u32(sdO), 16, 1024);
+        bool ok = mbar_wait(qdo_full, 0, abort_flag, p.guard, status_word(DQ_WIDE_KERNEL_ID, ROLE_MMA, 0xFFFF));
+        if (n_it == 0) ok = false;
+        auto issue_s = [&](int j) -> bool {        // S = Q K^T
+            const int sl = j & 1;
+            if (!mbar_wait(&k_full[sl], (j >> 1) & 1, abort_flag, p.guard, status_word(DQ_WIDE_KERNEL_ID, ROLE_MMA, j))) return false;
+            tc_fence_after_sync();
+            if (elect_one()) {
+                const uint64_t dKs = smem_desc_sw128(smem_u32(sK + sl * TILE64_BYTES), 16, 1024);
+#pragma unroll
+                for (int k = 0; k < WIDE_D / 16; ++k)
+                    if (k < kd)
+                        umma_ss(tmem_u, desc_advance(dQ0, (k / 4) * BOX128_BYTES + (k % 4) * 32),
+                                desc_advance(dKs, (k / 4) * BOX64_BYTES + (k % 4) * 32), IDESC_S, k > 0 ? 1u : 0u);
+                umma_commit(s_full);
+            }
+            __syncwarp();
+            return true;
+        };
+        auto issue_dp = [&](int j) -> bool {       // dP = dO V^T
+            if (!mbar_wait(v_full, j & 1, abort_flag, p.guard, status_word(DQ_WIDE_KERNEL_ID, ROLE_MMA, j))) return false;
+            tc_fence_after_sync();
+            if (elect_one()) {
+                const uint64_t dVs = smem_desc_sw128(smem_u32(sV), 16, 1024);
+#pragma unroll
+                for (int k = 0; k < WIDE_D / 16; ++k)
+                    if (k < kd)
+                        umma_ss(tmem_u + 64, desc_advance(dDO0, (k / 4) * BOX128_BYTES + (k % 4) * 32),
+                                desc_advance(dVs, (k / 4) * BOX64_BYTES + (k % 4) * 32), IDESC_S, k > 0 ? 1u : 0u);
+                umma_commit(dp_full);
+                umma_commit(v_empty);
+            }
+            __syncwarp();
+            return true;
+        };
+        if (ok) ok = issue_s(0);
+        if (ok) ok = issue_dp(0);
+        for (int j = 0; j < n_it && ok; ++j) {
+            const int sl = j & 1;
+            ok = mbar_wait(ds_ready, j & 1, abort_flag, p.guard, status_word(DQ_WIDE_KERNEL_ID, ROLE_MMA, j));
+            if (!ok) break;
+            tc_fence_after_sync();
+            if (elect_one()) {                     // dQ += dS K   (K read MN-major over all its column boxes)
+                const uint64_t dKm = smem_desc_sw128(smem_u32(sK + sl * TILE64_BYTES), BOX64_BYTES, 1024);
+#pragma unroll
+                for (int k = 0; k < WIDE_N / 16; ++k)
+                    umma_ts(tmem_u + 128, tmem_u + 64 + k * 8, desc_advance(dKm, k * 2048), IDESC_G, (j > 0 || k > 0) ? 1u : 0u);
+                umma_commit(&k_empty[sl]);
+                if (j == n_it - 1) umma_commit(final_bar);
+            }
+            __syncwarp();
+            if (j + 1 < n_it) {
+                ok = issue_s(j + 1);               // the scores of step j were read before dS(j) was signalled
+                if (!ok) break;
+                ok = issue_dp(j + 1);              // overwrites dS(j): ordered behind dQ(j)
+            }
+        }
+    } else if (warp >= 4) {
+        // compute: P (registers), dS; epilogue.  One thread per query row, 64 key columns per step.
+        const int quad = warp & 3;
+        const int r = quad * 32 + lane;
+        const int row = q0 + r;
+        const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
+        const uint32_t tS = tmem_base + lane_addr;
+        const uint32_t tDP = tmem_base + lane_addr + 64;
+        float lse2 = INFINITY, dl = 0.0f;          // rows past the end: P = 0
+        if (row < Sq && n_it > 0) {
+            const size_t idx = static_cast<size_t>(bh) * p.Sq + row;
+            lse2 = p.lse[idx] * LOG2E;
+            dl = p.delta[idx];
+        }
+        const float2 c2 = make_float2(p.scale_log2e, p.scale_log2e);
+        const float2 nl2 = make_float2(-lse2, -lse2);
+        const float2 ndl2 = make_float2(-dl, -dl);
+        bool ok = true;
+        for (int j = 0; j < n_it; ++j) {
+            ok = mbar_wait(s_full, j & 1, abort_flag, p.guard, status_word(DQ_WIDE_KERNEL_ID, ROLE_SOFTMAX, j));
+            if (!ok) break;
+            tc_fence_after_sync();
+            const int c0 = j * WIDE_N;
+            const bool need_mask = (c0 + WIDE_N > Sk) || (CAUSAL && (c0 + WIDE_N - 1 > q0 + off));
+            int limit = Sk - c0;
+            if (CAUSAL) limit = min(limit, row + off - c0 + 1);
+            float2 pr[32];
+            uint32_t sv[2][32];
+            tmem_ld32(tS, sv[0]);
+            tmem_ld32(tS + 32, sv[1]);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const int col = c * 32 + 2 * i;
+                    const float2 x = __ffma2_rn(make_float2(__uint_as_float(sv[c][2 * i]), __uint_as_float(sv[c][2 * i + 1])), c2, nl2);
+                    float2 e = prob_pair(i, x);
+                    if (need_mask) {
+                        if (col >= limit) e.x = 0.0f;
+                        if (col + 1 >= limit) e.y = 0.0f;
+                    }
+                    pr[c * 16 + i] = e;
+                }
+            }
+            ok = mbar_wait(dp_full, j & 1, abort_flag, p.guard, status_word(DQ_WIDE_KERNEL_ID, ROLE_SOFTMAX, j));
+            if (!ok) break;
+            tc_fence_after_sync();
+            tmem_ld32(tDP, sv[0]);
+            tmem_ld32(tDP + 32, sv[1]);
+            tmem_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 2; ++c) {
+                uint32_t dd[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float2 df = __fadd2_rn(make_float2(__uint_as_float(sv[c][2 * i]), __uint_as_float(sv[c][2 * i + 1])), ndl2);
+                    const float2 ds = __fmul2_rn(pr[c * 16 + i], df);
+                    dd[i] = pack16<F16>(ds.x, ds.y);
+                }
+                tmem_st16(tDP + c * 16, dd);
+            }
+            tmem_wait_st();
+            tc_fence_before_sync();
+            mbar_arrive(ds_ready);
+        }
+        __nv_bfloat16 *dq_row = p.dq + (static_cast<size_t>(bh) * p.Sq + row) * p.d;
+        if (n_it == 0) {
+            if (row < Sq)
+                for (int i = 0; i < p.d / 8; ++i) reinterpret_cast<uint4 *>(dq_row)[i] = make_uint4(0, 0, 0, 0);
+            ok = false;
+        }
+        if (ok) ok = mbar_wait(final_bar, 0, abort_flag, p.guard, status_word(DQ_WIDE_KERNEL_ID, ROLE_EPILOGUE, 0));
+        if (ok) {
+            tc_fence_after_sync();
+            uint8_t *scratch = sK + (warp - 4) * STORE_SCRATCH_BYTES;        // every product has completed: the K slots are free
+            const size_t stride = static_cast<size_t>(p.d);
+            __nv_bfloat16 *warp_dst = dq_row - static_cast<size_t>(lane) * stride;
+            const int rows_valid = min(32, Sq - (q0 + quad * 32));
+#pragma unroll
+            for (int c = 0; c < WIDE_D / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tmem_base + lane_addr + 128 + c * 32, v);
+                tmem_wait_ld();
+                store_rows16<F16>(warp_dst + c * 32, stride, v, p.scale, rows_valid, scratch, lane, p.d - c * 32);
+            }
+        }
+    }
+
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after_sync();
+        tmem_dealloc(tmem_base, L::TMEM_COLS);
+    }
+}
+
+template <bool CAUSAL, bool F16>
+static int launch_wide(const CUtensorMap &q64, const CUtensorMap &do64, const CUtensorMap &k128, const CUtensorMap &v128,
+                       const CUtensorMap &q128, const CUtensorMap &do128, const CUtensorMap &k64, const CUtensorMap &v64, BwdParams prm,
+                       const __nv_bfloat16 *o, const __nv_bfloat16 *d_o, float *delta, int B, cudaStream_t stream)
+{
+    static std::atomic<bool> configured[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaError_t e;
+    if (!configured[dev & 63].load(std::memory_order_acquire)) {
+        e = cudaFuncSetAttribute(bwd_dkdv_wide_kernel<CAUSAL, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, DkdvWideSmem::BYTES);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(dkdv wide)");
+        e = cudaFuncSetAttribute(bwd_dq_wide_kernel<CAUSAL, F16>, cudaFuncAttributeMaxDynamicSharedMemorySize, DqWideSmem::BYTES);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaFuncSetAttribute(dq wide)");
+        configured[dev & 63].store(true, std::memory_order_release);
+    }
+    const long long n_rows = static_cast<long long>(B) * prm.Hq * prm.Sq;
+    long long delta_blocks = (n_rows + 7) / 8;                         // 32 threads per row (d / 8 <= 32 pieces), 8 rows per block
+    if (delta_blocks > NUM_SMS * 32) delta_blocks = NUM_SMS * 32;
+    bwd_delta_kernel<32, F16><<<static_cast<int>(delta_blocks), 256, 0, stream>>>(o, d_o, delta, n_rows, 0, prm.d);
+    if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_delta_kernel launch");
+
+    prm.n_tiles = (prm.Sk + TILE - 1) / TILE;
+    const dim3 grid_kv(static_cast<unsigned>(prm.n_tiles * B * prm.Hkv), 2);
+    bwd_dkdv_wide_kernel<CAUSAL, F16><<<grid_kv, WIDE_THREADS, DkdvWideSmem::BYTES, stream>>>(q64, k128, v128, do64, prm);
+    if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_dkdv_wide_kernel launch");
+
+    prm.n_tiles = (prm.Sq + TILE - 1) / TILE;
+    bwd_dq_wide_kernel<CAUSAL, F16><<<prm.n_tiles * B * prm.Hq, WIDE_THREADS, DqWideSmem::BYTES, stream>>>(q128, k64, v64, do128, prm);
+    if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_dq_wide_kernel launch");
+    return VT_ATTN_OK;
+}
+
+int launch_bwd_wide(bool f16, const void *q, const void *k, const void *v, const void *o, const void *d_o, BwdParams prm, float *delta,
+                    int B, int causal, cudaStream_t stream)
+{
+    int rc;
+    CUtensorMap q64, do64, k128, v128, q128, do128, k64, v64;
+    const int D = prm.d, Sq = prm.Sq, Sk = prm.Sk;
+    if ((rc = make_tensor_map(&q64, q, B * prm.Hq, Sq, D, WIDE_N)) != VT_ATTN_OK) return rc;
+    if ((rc = make_tensor_map(&do64, d_o, B * prm.Hq, Sq, D, WIDE_N)) != VT_ATTN_OK) return rc;
+    if ((rc = make_tensor_map(&k128, k, B * prm.Hkv, Sk, D, TILE)) != VT_ATTN_OK) return rc;
+    if ((rc = make_tensor_map(&v128, v, B * prm.Hkv, Sk, D, TILE)) != VT_ATTN_OK) return rc;
+    if ((rc = make_tensor_map(&q128, q, B * prm.Hq, Sq, D, TILE)) != VT_ATTN_OK) return rc;
+    if ((rc = make_tensor_map(&do128, d_o, B * prm.Hq, Sq, D, TILE)) != VT_ATTN_OK) return rc;
+    if ((rc = make_tensor_map(&k64, k, B * prm.Hkv, Sk, D, WIDE_N)) != VT_ATTN_OK) return rc;
+    if ((rc = make_tensor_map(&v64, v, B * prm.Hkv, Sk, D, WIDE_N)) != VT_ATTN_OK) return rc;
+    const __nv_bfloat16 *o_ = static_cast<const __nv_bfloat16 *>(o), *do_ = static_cast<const __nv_bfloat16 *>(d_o);
+    if (f16)
+        return causal ? launch_wide<true, true>(q64, do64, k128, v128, q128, do128, k64, v64, prm, o_, do_, delta, B, stream)
+                      : launch_wide<false, true>(q64, do64, k128, v128, q128, do128, k64, v64, prm, o_, do_, delta, B, stream);
+    return causal ? launch_wide<true, false>(q64, do64, k128, v128, q128, do128, k64, v64, prm, o_, do_, delta, B, stream)
+                  : launch_wide<false, false>(q64, do64, k128, v128, q128, do128, k64, v64, prm, o_, do_, delta, B, stream);
+}
+
+}  // namespace vt

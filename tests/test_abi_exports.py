@@ -95,7 +95,8 @@ def test_workspace_and_staging_sizes(lib):
     assert vt.vt_attn_bwd_workspace_bytes(1, 3, 2, 128, 128, 64) == 0       # Hq % Hkv != 0
     assert vt.vt_attn_bwd_workspace_bytes(1, 2, 2, 128, 128, 100) == 0      # unsupported D (not a multiple of 8)
     assert vt.vt_attn_bwd_workspace_bytes(1, 2, 2, 128, 128, 96) == 1024     # any multiple of 8 up to 128
-    assert vt.vt_attn_bwd_workspace_bytes(1, 2, 2, 128, 128, 136) == 0
+    assert vt.vt_attn_bwd_workspace_bytes(1, 2, 2, 128, 128, 136) == 1024    # and up to 256
+    assert vt.vt_attn_bwd_workspace_bytes(1, 2, 2, 128, 128, 264) == 0
     assert vt.vt_attn_fwd_kernel_kind(1, 2, 2, 128, 128, 256, False) == 0       # forward only: up to 256
     assert vt.vt_attn_fwd_splitkv_plan(1, 8, 2, 1, 4096, 256)[0] >= 1
     # packed batches: equal cache lengths get the one-wave choice of the batched call, ragged ones more chunks
@@ -141,12 +142,16 @@ def test_argument_validation_returns_before_any_cuda_call(lib):
     assert g(*args, None, 4096, None) == vt.ERR_INVALID_ARGUMENT
     bad = [_fake()] * 9 + [1, 2, 2, 128, 128, 84, 0, 0.125]
     assert g(*bad, _fake(), 4096, None) == vt.ERR_UNSUPPORTED
-    bad = [_fake()] * 9 + [1, 2, 2, 128, 128, 192, 0, 0.125]         # the backward stops at 128
+    bad = [_fake()] * 9 + [1, 2, 2, 128, 128, 264, 0, 0.125]         # the backward goes up to 256 too
     assert g(*bad, _fake(), 4096, None) == vt.ERR_UNSUPPORTED
+    wide = [_fake()] * 9 + [1, 2, 2, 128, 128, 192, 0, 0.125]
+    assert g(*wide, _fake(), 16, None) == vt.ERR_WORKSPACE_TOO_SMALL  # 128 < D <= 256 is accepted: the next check answers
+    assert vt.vt_attn_bwd_kernel_kind(1, 2, 2, 128, 128, 192) == 2 and vt.vt_attn_bwd_kernel_kind(1, 2, 2, 128, 128, 128) == 0
+    assert vt.vt_attn_bwd_workspace_bytes(1, 2, 2, 128, 128, 256) == 1024
     assert lib.vt_attn_fwd_host(*([_fake()] * 5), 1, 2, 2, 128, 128, 64, 0, 0.125, _fake(0x10000), 16, None) \
         == vt.ERR_WORKSPACE_TOO_SMALL
     assert lib.vt_attn_selftest_timeout(0, None) == vt.ERR_INVALID_ARGUMENT
-    # head dimensions above 128 exist only in the [B, H, S, D] forward entry points: the packed ones and the host-buffer
+    # head dimensions above 128 exist only in the [B, H, S, D] forward and backward entry points: the packed ones and the host-buffer
     # ones answer "unsupported", as does a V width outside [8, 256]
     cu = _fake(0x2000)
     assert lib.vt_attn_fwd_varlen(*([_fake()] * 5), cu, cu, 2, 2, 2, 256, 256, 128, 128, 192, 0, 0.1, None) == vt.ERR_UNSUPPORTED

@@ -1,0 +1,66 @@
+"""GPU: the backward for head dimensions above 128 (up to 256): Delta, a dK/dV kernel that keeps 128 keys x 256 columns
+stationary and walks the queries 64 at a time (twice: one half of the output columns per pass), and a dQ kernel that
+keeps 128 queries stationary and walks the keys 64 at a time - against the fp64 oracle, element by element."""
+import numpy as np
+import pytest
+
+from helpers import check_fwd, check_grad, dev, host
+from oracle import attn_oracle as orc
+from paper_2601_16238_b200.inputs import AttnConfig, make_inputs
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [
+    # B, Hq, Hkv, Sq, Sk, D, causal
+    (1, 1, 1, 128, 128, 256, 0),
+    (1, 2, 2, 64, 64, 256, 1),
+    (1, 2, 1, 200, 333, 256, 0),          # ragged ends, two heads per KV head
+    (2, 4, 2, 300, 300, 192, 1),          # the other common size: the second column half holds 64 columns
+    (1, 2, 2, 257, 129, 136, 1),          # eight columns in the second half; top-left mask with Sq > Sk
+    (1, 2, 1, 190, 450, 256, 2),          # bottom-right aligned mask
+    (1, 2, 2, 450, 190, 200, 2),          # fewer keys than queries: leading rows see nothing
+    (1, 3, 3, 1, 1, 256, 1),
+    (1, 2, 2, 640, 640, 256, 1),
+]
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,D,causal", SHAPES)
+def test_backward_above_128_columns_matches_the_oracle(vt, B, Hq, Hkv, Sq, Sk, D, causal):
+    import torch
+    cfg = AttnConfig("wide", 24, B, Hq, Hkv, Sq, Sk, D, causal, True)
+    q, k, v, d_o = make_inputs(cfg)
+    tq, tk, tv, tdo = dev(q), dev(k), dev(v), dev(d_o)
+    assert vt.vt_attn_bwd_kernel_kind(B, Hq, Hkv, Sq, Sk, D) == 2
+    o, lse = vt.vt_attn_fwd(tq, tk, tv, causal, cfg.scale)
+    dq, dk, dv = (torch.full_like(t, float("nan")) for t in (tq, tk, tv))
+    ws = torch.full((max(64, vt.vt_attn_bwd_workspace_bytes(B, Hq, Hkv, Sq, Sk, D) // 4),), float("nan"), device="cuda").view(torch.uint8)
+    vt.vt_attn_bwd(tq, tk, tv, o, tdo, lse, causal, cfg.scale, dq, dk, dv, ws)
+    again = vt.vt_attn_bwd(tq, tk, tv, o, tdo, lse, causal, cfg.scale)
+    torch.cuda.synchronize()
+    rc, detail = vt.vt_attn_device_status()
+    assert rc == 0, f"device status {rc} detail {detail:#x}"
+    for a, b in zip((dq, dk, dv), again):
+        assert torch.equal(a, b)
+    o_ref, lse_ref = orc.attn_fwd(q, k, v, causal, cfg.scale)
+    finite = np.isfinite(lse_ref)
+    assert np.abs(host(o) - o_ref).max() <= max(1e-2, 2.0 ** -8 * np.abs(o_ref).max())
+    assert (np.abs(host(lse)[finite] - lse_ref[finite]) <= 1e-3 * np.maximum(1.0, np.abs(lse_ref[finite]))).all()
+    refs = orc.attn_bwd(q, k, v, d_o, causal, cfg.scale)
+    for name, a, ref in zip(("dQ", "dK", "dV"), (dq, dk, dv), refs):
+        check_grad(host(a), ref, name, f"wide {cfg}")
+
+
+def test_backward_above_128_columns_fp16(vt):
+    import torch
+    from paper_2601_16238_b200.inputs import normal_f16
+    B, Hq, Hkv, Sq, Sk, D, causal = 1, 4, 2, 260, 390, 256, 1
+    scale = float(np.float32(1.0) / np.sqrt(np.float32(D)))
+    bits = [normal_f16(s, 9470 + i) for i, s in enumerate(((B, Hq, Sq, D), (B, Hkv, Sk, D), (B, Hkv, Sk, D), (B, Hq, Sq, D)))]
+    q, k, v, d_o = (torch.from_numpy(np.ascontiguousarray(x).view(np.int16)).view(torch.float16).cuda() for x in bits)
+    o, lse = vt.vt_attn_fwd_f16(q, k, v, causal, scale)
+    got = vt.vt_attn_bwd_f16(q, k, v, o, d_o, lse, causal, scale)
+    torch.cuda.synchronize()
+    assert vt.vt_attn_device_status()[0] == 0
+    refs = orc.attn_bwd(*(orc.f16_bits_to_f64(x) for x in bits), causal, scale)
+    for name, a, ref in zip(("dQ", "dK", "dV"), got, refs):
+        check_grad(host(a), ref, name, "wide fp16")
