@@ -238,6 +238,26 @@ int vt_attn_fwd_dv_f16(const void *q, const void *k, const void *v, void *o, flo
                        int causal, float scale, void *stream);
 
 /*
+ * The backward of vt_attn_fwd_dv: V, O, dO and dV have Dv columns, Q, K, dQ and dK have D (both
+ * multiples of 8 up to 256, e.g. 192 / 128; the paper has no counterpart).  Same formulas,
+ * buffers and workspace (vt_attn_bwd_workspace_bytes(B, Hq, Hkv, Sq, Sk, D)) as vt_attn_bwd, to
+ * which the call forwards when Dv == D; other pairs run in the kernels built for head
+ * dimensions above 128 (vt_attn_bwd_kernel_kind 2), whatever their size.
+ */
+int vt_attn_bwd_dv(const void *q, const void *k, const void *v,
+                   const void *o, const void *d_o, const float *lse,
+                   void *dq, void *dk, void *dv,
+                   int B, int Hq, int Hkv, int Sq, int Sk, int D, int Dv,
+                   int causal, float scale,
+                   void *workspace, size_t workspace_bytes, void *stream);
+int vt_attn_bwd_dv_f16(const void *q, const void *k, const void *v,
+                       const void *o, const void *d_o, const float *lse,
+                       void *dq, void *dk, void *dv,
+                       int B, int Hq, int Hkv, int Sq, int Sk, int D, int Dv,
+                       int causal, float scale,
+                       void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Which forward kernel vt_attn_fwd / vt_attn_fwd_f16 launch for a shape: 0 the one-tile kernel
  * (one 128-row query tile per block, 64-key steps), 1 the two-tile kernel (two query tiles per
  * block side by side, 128-key steps; long D = 128 sequences), 2 the one-tile kernel run over a

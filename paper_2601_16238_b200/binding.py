@@ -37,6 +37,8 @@ EXPORTS = {
     "vt_attn_fwd_kernel_kind": (_i, _DIMS + [_i]),
     "vt_attn_fwd_f16": (_i, [_vp] * 5 + _DIMS + [_i, _f, _vp]),
     "vt_attn_bwd_f16": (_i, [_vp] * 9 + _DIMS + [_i, _f, _vp, _sz, _vp]),
+    "vt_attn_bwd_dv": (_i, [_vp] * 9 + _DIMS + [_i, _i, _f, _vp, _sz, _vp]),
+    "vt_attn_bwd_dv_f16": (_i, [_vp] * 9 + _DIMS + [_i, _i, _f, _vp, _sz, _vp]),
     "vt_attn_bwd_workspace_bytes": (_sz, _DIMS),
     "vt_attn_bwd_kernel_kind": (_i, _DIMS),
     "vt_attn_bwd": (_i, [_vp] * 9 + _DIMS + [_i, _f, _vp, _sz, _vp]),
@@ -357,6 +359,35 @@ def vt_attn_bwd_f16(q, k, v, o, d_o, lse, causal: bool, scale: float, dq=None, d
     """Backward attention on fp16 tensors.  Returns (dQ, dK, dV) in fp16."""
     import torch
     return _bwd("vt_attn_bwd_f16", torch.float16, q, k, v, o, d_o, lse, causal, scale, dq, dk, dv, workspace, stream)
+
+
+def _bwd_dv(entry: str, dtype, q, k, v, o, d_o, lse, causal, scale, dq, dk, dv, workspace, stream):
+    import torch
+    lib = load_library()
+    dims = _dims(q, k, v, own_dv=True)
+    Dv = int(v.shape[-1])
+    o_shape = tuple(q.shape[:3]) + (Dv,)
+    _shapes((o, "o", o_shape), (d_o, "d_o", o_shape), (lse, "lse", q.shape[:3]), (dq, "dq", q.shape), (dk, "dk", k.shape), (dv, "dv", v.shape))
+    _inputs(dtype, "cuda", q, k=k, v=v, o=o, d_o=d_o)
+    _require(lse, torch.float32, "lse", device=q.device)
+    dq, dk, dv = _grad_out(dq, q, "dq"), _grad_out(dk, k, "dk"), _grad_out(dv, v, "dv")
+    workspace = _workspace(workspace, 0 if workspace is not None else lib.vt_attn_bwd_workspace_bytes(*dims), q.device)
+    rc = _call(q.device, getattr(lib, entry), _p(q), _p(k), _p(v), _p(o), _p(d_o), _p(lse), _p(dq), _p(dk), _p(dv), *dims, Dv,
+               _mask_mode(causal), float(scale), _p(workspace), workspace.numel() * workspace.element_size(), _stream(stream, q.device))
+    _check(rc, entry)
+    return dq, dk, dv
+
+
+def vt_attn_bwd_dv(q, k, v, o, d_o, lse, causal, scale: float, dq=None, dk=None, dv=None, workspace=None, stream=None):
+    """Backward of vt_attn_fwd_dv: q, k [B,H,S,D], v, o, d_o [.., Dv] (bf16).  Returns (dQ, dK, dV)."""
+    import torch
+    return _bwd_dv("vt_attn_bwd_dv", torch.bfloat16, q, k, v, o, d_o, lse, causal, scale, dq, dk, dv, workspace, stream)
+
+
+def vt_attn_bwd_dv_f16(q, k, v, o, d_o, lse, causal, scale: float, dq=None, dk=None, dv=None, workspace=None, stream=None):
+    """vt_attn_bwd_dv on fp16 tensors."""
+    import torch
+    return _bwd_dv("vt_attn_bwd_dv_f16", torch.float16, q, k, v, o, d_o, lse, causal, scale, dq, dk, dv, workspace, stream)
 
 
 def _bwd_static(name, dtype, q, k, v, o, d_o, lse, causal, scale, dq, dk, dv, stream):

@@ -1016,6 +1016,66 @@ extern "C" int vt_attn_bwd_f16(const void *q, const void *k, const void *v, cons
     return bwd_entry(true, q, k, v, o, d_o, lse, dq, dk, dv, B, Hq, Hkv, Sq, Sk, D, causal, scale, workspace, workspace_bytes, stream);
 }
 
+// Backward with V (and O, dO, dV) of their own width: the kernels of bwd_wide.cu, which take the two widths separately.
+static int bwd_dv_entry(bool f16, const void *q, const void *k, const void *v, const void *o, const void *d_o, const float *lse,
+                        void *dq, void *dk, void *dv, int B, int Hq, int Hkv, int Sq, int Sk, int D, int Dv, int causal,
+                        float scale, void *workspace, size_t workspace_bytes, void *stream)
+{
+    using namespace vt;
+    if (D == Dv) return bwd_entry(f16, q, k, v, o, d_o, lse, dq, dk, dv, B, Hq, Hkv, Sq, Sk, D, causal, scale, workspace, workspace_bytes, stream);
+    Shape s{B, Hq, Hkv, Sq, Sk, D};
+    int rc = check_shape(s, scale, MAX_HEAD_DIM_FWD);
+    if (rc != VT_ATTN_OK) return rc;
+    if (!head_dim_ok(Dv, MAX_HEAD_DIM_FWD)) return VT_ATTN_ERR_UNSUPPORTED;
+    if (!ptr_ok(q) || !ptr_ok(k) || !ptr_ok(v) || !ptr_ok(o) || !ptr_ok(d_o) || !ptr_ok(lse, 4) || !ptr_ok(dq) ||
+        !ptr_ok(dk) || !ptr_ok(dv) || !ptr_ok(workspace))
+        return VT_ATTN_ERR_INVALID_ARGUMENT;
+    if (workspace_bytes < align256(static_cast<size_t>(B) * Hq * Sq * sizeof(float))) return VT_ATTN_ERR_WORKSPACE_TOO_SMALL;
+    if (causal < 0 || causal > 2) return VT_ATTN_ERR_INVALID_ARGUMENT;
+    rc = check_device();
+    if (rc != VT_ATTN_OK) return rc;
+    const long long max_blocks = static_cast<long long>((Sq > Sk ? Sq : Sk) + TILE - 1) / TILE * B * Hq;
+    if (max_blocks > 0x7FFFFFFFll) return VT_ATTN_ERR_INVALID_ARGUMENT;
+    BwdParams prm;
+    prm.lse = lse;
+    prm.delta = static_cast<float *>(workspace);
+    prm.dq = static_cast<__nv_bfloat16 *>(dq);
+    prm.dk = static_cast<__nv_bfloat16 *>(dk);
+    prm.dv = static_cast<__nv_bfloat16 *>(dv);
+    prm.Hq = Hq;
+    prm.Hkv = Hkv;
+    prm.d = D;
+    prm.d_v = Dv;
+    prm.G = Hq / Hkv;
+    prm.Sq = Sq;
+    prm.Sk = Sk;
+    prm.n_tiles = 0;
+    prm.cu_q = nullptr;
+    prm.cu_k = nullptr;
+    prm.total_q = 0;
+    prm.bottom_right = (causal == 2);
+    prm.head_group = 0;
+    prm.scale = scale;
+    prm.scale_log2e = scale * LOG2E;
+    prm.guard = make_guard();
+    if (!prm.guard.status) return VT_ATTN_ERR_CUDA;
+    return launch_bwd_wide(f16, q, k, v, o, d_o, prm, static_cast<float *>(workspace), B, causal, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int vt_attn_bwd_dv(const void *q, const void *k, const void *v, const void *o, const void *d_o, const float *lse,
+                              void *dq, void *dk, void *dv, int B, int Hq, int Hkv, int Sq, int Sk, int D, int Dv, int causal,
+                              float scale, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return bwd_dv_entry(false, q, k, v, o, d_o, lse, dq, dk, dv, B, Hq, Hkv, Sq, Sk, D, Dv, causal, scale, workspace, workspace_bytes, stream);
+}
+
+extern "C" int vt_attn_bwd_dv_f16(const void *q, const void *k, const void *v, const void *o, const void *d_o, const float *lse,
+                                  void *dq, void *dk, void *dv, int B, int Hq, int Hkv, int Sq, int Sk, int D, int Dv, int causal,
+                                  float scale, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return bwd_dv_entry(true, q, k, v, o, d_o, lse, dq, dk, dv, B, Hq, Hkv, Sq, Sk, D, Dv, causal, scale, workspace, workspace_bytes, stream);
+}
+
 extern "C" size_t vt_attn_bwd_varlen_workspace_bytes(int Hq, int total_q)
 {
     if (Hq <= 0 || total_q <= 0) return 0;

@@ -64,6 +64,7 @@ struct BwdParams {
     __nv_bfloat16 *dq, *dk, *dv;
     int Hq, Hkv, G, Sq, Sk;
     int d;                  // head dimension of the tensors in global memory (<= the kernels' D; the columns between read as zero)
+    int d_v = 0;            // bwd_wide.cu only: head dimension of V, O, dO, dV when it differs from that of Q, K, dQ, dK (0: the same)
     int n_tiles;            // tiles per head along the block's stationary dimension (of the longest sequence)
     float scale, scale_log2e;
     const int *cu_q;        // packed batches only: cumulative sequence lengths [n_seqs + 1], device

@@ -95,8 +95,11 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const int qt_start = CAUSAL ? min(max(k0 - off, 0) / WIDE_N, n_qt) : 0;   // first query tile with a query that sees key k0
     const int n_qi = n_qt - qt_start;
     const int n_it = n_qi * p.G;
-    const int cols_out = min(TILE, p.d - half * TILE);    // real columns of this half (> 0: d > 128)
-    const int kd = (p.d + 15) >> 4;                       // 16-column contraction steps that hold data
+    const int dv_w = p.d_v > 0 ? p.d_v : p.d;             // width of V, dO, dV (Q, K, dK: p.d)
+    const int cols_k = min(TILE, p.d - half * TILE);      // real columns of dK in this half (<= 0: none)
+    const int cols_v = min(TILE, dv_w - half * TILE);     // of dV
+    const int kd = (p.d + 15) >> 4;                       // 16-column contraction steps of S^T = K Q^T that hold data
+    const int kdv = (dv_w + 15) >> 4;                     // of dP^T = V dO^T
 
     if (threadIdx.x == 0) {
         mbar_init(kv_full, 1);
@@ -189,7 +192,8 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     } else if (warp == 1) {
         // MMA issuer.  Per iteration: dV(i), S(i+1), dK(i), dP(i+1) - the order of the 128-column kernel.
         constexpr uint32_t IDESC_S = make_idesc(128, WIDE_N, fmt16<F16>(), fmt16<F16>(), 0, 0);
-        const uint32_t IDESC_G = make_idesc(128, ((cols_out + 15) >> 4) * 16, fmt16<F16>(), fmt16<F16>(), 0, 1);
+        const uint32_t IDESC_GV = make_idesc(128, ((max(cols_v, 8) + 15) >> 4) * 16, fmt16<F16>(), fmt16<F16>(), 0, 1);
+        const uint32_t IDESC_GK = make_idesc(128, ((max(cols_k, 8) + 15) >> 4) * 16, fmt16<F16>(), fmt16<F16>(), 0, 1);
         const uint32_t tmem_u = __shfl_sync(0xFFFFFFFFu, tmem_base, 0);
         const uint64_t dK0 = smem_desc_sw128(smem_u32(sK), 16, 1024), dV0 = smem_desc_sw128(smem_u32(sV), 16, 1024);
         // dO and Q as MN-major B operands restricted to this block's column half: boxes 2 * half and 2 * half + 1
@@ -218,7 +222,7 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 const uint64_t dDOs = smem_desc_sw128(smem_u32(sdO), 16, 1024);
 #pragma unroll
                 for (int k = 0; k < WIDE_D / 16; ++k)
-                    if (k < kd)
+                    if (k < kdv)
                         umma_ss(tmem_u + 64, desc_advance(dV0, (k / 4) * BOX128_BYTES + (k % 4) * 32),
                                 desc_advance(dDOs, (k / 4) * BOX64_BYTES + (k % 4) * 32), IDESC_S, k > 0 ? 1u : 0u);
                 umma_commit(dp_full);
@@ -234,9 +238,11 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             if (!ok) break;
             tc_fence_after_sync();
             if (elect_one()) {                     // dV[:, half] += P^T dO[:, half]   (16 query rows per instruction)
+                if (cols_v > 0) {
 #pragma unroll
-                for (int k = 0; k < WIDE_N / 16; ++k)
-                    umma_ts(tmem_u + 128, tmem_u + k * 8, desc_advance(dDOm, k * 2048), IDESC_G, (it > 0 || k > 0) ? 1u : 0u);
+                    for (int k = 0; k < WIDE_N / 16; ++k)
+                        umma_ts(tmem_u + 128, tmem_u + k * 8, desc_advance(dDOm, k * 2048), IDESC_GV, (it > 0 || k > 0) ? 1u : 0u);
+                }
                 umma_commit(do_empty);
             }
             __syncwarp();
@@ -249,9 +255,11 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             tc_fence_after_sync();
             if (elect_one()) {                     // dK[:, half] += dS^T Q[:, half]
                 const uint64_t dQm = smem_desc_sw128(smem_u32(sQ + sl * TILE64_BYTES + half * 2 * BOX64_BYTES), BOX64_BYTES, 1024);
+                if (cols_k > 0) {
 #pragma unroll
-                for (int k = 0; k < WIDE_N / 16; ++k)
-                    umma_ts(tmem_u + 256, tmem_u + 64 + k * 8, desc_advance(dQm, k * 2048), IDESC_G, (it > 0 || k > 0) ? 1u : 0u);
+                    for (int k = 0; k < WIDE_N / 16; ++k)
+                        umma_ts(tmem_u + 256, tmem_u + 64 + k * 8, desc_advance(dQm, k * 2048), IDESC_GK, (it > 0 || k > 0) ? 1u : 0u);
+                }
                 umma_commit(&q_empty[sl]);
                 if (it == n_it - 1) umma_commit(final_bar);
             }
@@ -342,26 +350,28 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             if (lane == 0) mbar_arrive(&rows_empty[rsl]);
         }
         // epilogue: this block's column half of dV, then of dK
-        const size_t row_off = (static_cast<size_t>(bh_kv) * p.Sk + kv) * p.d + half * TILE;
+        const size_t row_v = (static_cast<size_t>(bh_kv) * p.Sk + kv) * dv_w + half * TILE;
+        const size_t row_k = (static_cast<size_t>(bh_kv) * p.Sk + kv) * p.d + half * TILE;
         if (n_it == 0) {
-            if (kv < Sk)
-                for (int i = 0; i < cols_out / 8; ++i) {
-                    reinterpret_cast<uint4 *>(p.dv + row_off)[i] = make_uint4(0, 0, 0, 0);
-                    reinterpret_cast<uint4 *>(p.dk + row_off)[i] = make_uint4(0, 0, 0, 0);
-                }
+            if (kv < Sk) {
+                for (int i = 0; i < cols_v / 8; ++i) reinterpret_cast<uint4 *>(p.dv + row_v)[i] = make_uint4(0, 0, 0, 0);
+                for (int i = 0; i < cols_k / 8; ++i) reinterpret_cast<uint4 *>(p.dk + row_k)[i] = make_uint4(0, 0, 0, 0);
+            }
         } else {
             if (ok) ok = mbar_wait(final_bar, 0, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_EPILOGUE, 0));
             if (ok) {
                 tc_fence_after_sync();
                 uint8_t *scratch = sQ + (warp - 4) * STORE_SCRATCH_BYTES;     // every product has completed: the Q slots are free
                 const int row0 = k0 + quad * 32;
-                const size_t stride = static_cast<size_t>(p.d);
                 const int rows_valid = min(32, Sk - row0);
 #pragma unroll
                 for (int t = 0; t < 2; ++t) {
-                    __nv_bfloat16 *warp_dst = (t == 0 ? p.dv : p.dk) + row_off - static_cast<size_t>(lane) * stride;
+                    const size_t stride = static_cast<size_t>(t == 0 ? dv_w : p.d);
+                    const int cols_out = (t == 0) ? cols_v : cols_k;
+                    __nv_bfloat16 *warp_dst = (t == 0 ? p.dv + row_v : p.dk + row_k) - static_cast<size_t>(lane) * stride;
                     const uint32_t tSrc = tmem_base + lane_addr + 128 + t * 128;
                     const float mul = (t == 0) ? 1.0f : p.scale;
+                    if (cols_out <= 0) continue;                       // this half holds no column of the tensor (block-uniform)
 #pragma unroll
                     for (int c = 0; c < TILE / 32; ++c) {
                         uint32_t v[32];
@@ -439,7 +449,8 @@ bwd_dq_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
     const int off = (CAUSAL && p.bottom_right) ? Sk - Sq : 0;
     int n_it = (Sk + WIDE_N - 1) / WIDE_N;                 // steps of 64 keys
     if (CAUSAL) n_it = (q0 + TILE - 1 + off < 0) ? 0 : min(n_it, (q0 + TILE - 1 + off) / WIDE_N + 1);
-    const int kd = (p.d + 15) >> 4;
+    const int kd = (p.d + 15) >> 4;                                   // contraction steps of S = Q K^T (and N / 16 of dQ)
+    const int kdv = ((p.d_v > 0 ? p.d_v : p.d) + 15) >> 4;             // of dP = dO V^T
 
     if (threadIdx.x == 0) {
         mbar_init(qdo_full, 1);
@@ -527,7 +538,7 @@ bwd_dq_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_consta
                 const uint64_t dVs = smem_desc_sw128(smem_u32(sV), 16, 1024);
 #pragma unroll
                 for (int k = 0; k < WIDE_D / 16; ++k)
-                    if (k < kd)
+                    if (k < kdv)
                         umma_ss(tmem_u + 64, desc_advance(dDO0, (k / 4) * BOX128_BYTES + (k % 4) * 32),
                                 desc_advance(dVs, (k / 4) * BOX64_BYTES + (k % 4) * 32), IDESC_S, k > 0 ? 1u : 0u);
                 umma_commit(dp_full);
@@ -674,11 +685,12 @@ static int launch_wide(const CUtensorMap &q64, const CUtensorMap &do64, const CU
     const long long n_rows = static_cast<long long>(B) * prm.Hq * prm.Sq;
     long long delta_blocks = (n_rows + 7) / 8;                         // 32 threads per row (d / 8 <= 32 pieces), 8 rows per block
     if (delta_blocks > NUM_SMS * 32) delta_blocks = NUM_SMS * 32;
-    bwd_delta_kernel<32, F16><<<static_cast<int>(delta_blocks), 256, 0, stream>>>(o, d_o, delta, n_rows, 0, prm.d);
+    bwd_delta_kernel<32, F16><<<static_cast<int>(delta_blocks), 256, 0, stream>>>(o, d_o, delta, n_rows, 0, prm.d_v > 0 ? prm.d_v : prm.d);
     if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_delta_kernel launch");
 
     prm.n_tiles = (prm.Sk + TILE - 1) / TILE;
-    const dim3 grid_kv(static_cast<unsigned>(prm.n_tiles * B * prm.Hkv), 2);
+    const int widest = prm.d > prm.d_v ? prm.d : prm.d_v;
+    const dim3 grid_kv(static_cast<unsigned>(prm.n_tiles * B * prm.Hkv), widest > TILE ? 2 : 1);      // one pass per 128 columns of dK / dV
     bwd_dkdv_wide_kernel<CAUSAL, F16><<<grid_kv, WIDE_THREADS, DkdvWideSmem::BYTES, stream>>>(q64, k128, v128, do64, prm);
     if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_dkdv_wide_kernel launch");
 
@@ -693,15 +705,15 @@ int launch_bwd_wide(bool f16, const void *q, const void *k, const void *v, const
 {
     int rc;
     CUtensorMap q64, do64, k128, v128, q128, do128, k64, v64;
-    const int D = prm.d, Sq = prm.Sq, Sk = prm.Sk;
+    const int D = prm.d, Dv = prm.d_v > 0 ? prm.d_v : prm.d, Sq = prm.Sq, Sk = prm.Sk;
     if ((rc = make_tensor_map(&q64, q, B * prm.Hq, Sq, D, WIDE_N)) != VT_ATTN_OK) return rc;
-    if ((rc = make_tensor_map(&do64, d_o, B * prm.Hq, Sq, D, WIDE_N)) != VT_ATTN_OK) return rc;
+    if ((rc = make_tensor_map(&do64, d_o, B * prm.Hq, Sq, Dv, WIDE_N)) != VT_ATTN_OK) return rc;
     if ((rc = make_tensor_map(&k128, k, B * prm.Hkv, Sk, D, TILE)) != VT_ATTN_OK) return rc;
-    if ((rc = make_tensor_map(&v128, v, B * prm.Hkv, Sk, D, TILE)) != VT_ATTN_OK) return rc;
+    if ((rc = make_tensor_map(&v128, v, B * prm.Hkv, Sk, Dv, TILE)) != VT_ATTN_OK) return rc;
     if ((rc = make_tensor_map(&q128, q, B * prm.Hq, Sq, D, TILE)) != VT_ATTN_OK) return rc;
-    if ((rc = make_tensor_map(&do128, d_o, B * prm.Hq, Sq, D, TILE)) != VT_ATTN_OK) return rc;
+    if ((rc = make_tensor_map(&do128, d_o, B * prm.Hq, Sq, Dv, TILE)) != VT_ATTN_OK) return rc;
     if ((rc = make_tensor_map(&k64, k, B * prm.Hkv, Sk, D, WIDE_N)) != VT_ATTN_OK) return rc;
-    if ((rc = make_tensor_map(&v64, v, B * prm.Hkv, Sk, D, WIDE_N)) != VT_ATTN_OK) return rc;
+    if ((rc = make_tensor_map(&v64, v, B * prm.Hkv, Sk, Dv, WIDE_N)) != VT_ATTN_OK) return rc;
     const __nv_bfloat16 *o_ = static_cast<const __nv_bfloat16 *>(o), *do_ = static_cast<const __nv_bfloat16 *>(d_o);
     if (f16)
         return causal ? launch_wide<true, true>(q64, do64, k128, v128, q128, do128, k64, v64, prm, o_, do_, delta, B, stream)

@@ -64,3 +64,30 @@ def test_backward_above_128_columns_fp16(vt):
     refs = orc.attn_bwd(*(orc.f16_bits_to_f64(x) for x in bits), causal, scale)
     for name, a, ref in zip(("dQ", "dK", "dV"), got, refs):
         check_grad(host(a), ref, name, "wide fp16")
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,D,Dv,causal", [
+    (1, 4, 2, 300, 300, 192, 128, 1),      # the 192 / 128 pair
+    (2, 2, 2, 200, 333, 128, 256, 0),      # V wider than Q / K
+    (1, 2, 1, 129, 257, 64, 128, 2),       # both within 128 columns: still the kernels that take two widths
+    (1, 2, 2, 260, 260, 256, 72, 1),
+])
+def test_backward_with_v_of_its_own_width(vt, B, Hq, Hkv, Sq, Sk, D, Dv, causal):
+    """vt_attn_bwd_dv against the oracle on tensors padded with zero columns to a common width: zero columns of Q and K
+    add nothing to the scores and get zero gradients, zero columns of V and dO give zero columns of dV."""
+    import torch
+    from paper_2601_16238_b200.inputs import normal_bf16
+    scale = float(np.float32(1.0) / np.sqrt(np.float32(D)))
+    q, k, v, d_o = (normal_bf16(s, 9500 + i) for i, s in enumerate(((B, Hq, Sq, D), (B, Hkv, Sk, D), (B, Hkv, Sk, Dv), (B, Hq, Sq, Dv))))
+    tq, tk, tv, tdo = dev(q), dev(k), dev(v), dev(d_o)
+    o, lse = vt.vt_attn_fwd_dv(tq, tk, tv, causal, scale)
+    dq, dk, dv = vt.vt_attn_bwd_dv(tq, tk, tv, o, tdo, lse, causal, scale)
+    torch.cuda.synchronize()
+    assert vt.vt_attn_device_status()[0] == 0
+    assert dq.shape == tq.shape and dk.shape == tk.shape and dv.shape == tv.shape
+    W = max(D, Dv)
+    pad = lambda bits, w: np.concatenate([orc.bf16_bits_to_f64(bits), np.zeros(bits.shape[:3] + (W - w,))], axis=-1)      # noqa: E731
+    gq, gk, gv = orc.attn_bwd(pad(q, D), pad(k, D), pad(v, Dv), pad(d_o, Dv), causal, scale)
+    assert (gq[..., D:] == 0).all() and (gk[..., D:] == 0).all() and (gv[..., Dv:] == 0).all()
+    for name, a, ref in (("dQ", dq, gq[..., :D]), ("dK", dk, gk[..., :D]), ("dV", dv, gv[..., :Dv])):
+        check_grad(host(a), ref, name, f"D={D} Dv={Dv}")
