@@ -51,6 +51,54 @@ def test_random_shapes_forward_and_backward(vt, B, Hq, Hkv, Sq, Sk, D, causal, s
         assert np.abs(a - b).max() <= TOL_GRAD * np.abs(b).max() + 1e-5, nm
 
 
+def _wide_cases(n, seed):
+    return [c[:5] + (136 + 8 * (c[7] * 7 % 16),) + c[6:] for c in _cases(n, seed, 128)]      # D in 136 .. 256
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,D,causal,seed", _wide_cases(16, 5))
+def test_random_shapes_backward_above_128_columns(vt, B, Hq, Hkv, Sq, Sk, D, causal, seed):
+    import torch
+    cfg = AttnConfig("fuzz_wide", seed, B, Hq, Hkv, Sq, Sk, D, causal, True)
+    q, k, v, d_o = make_inputs(cfg)
+    tq, tk, tv, tdo = dev(q), dev(k), dev(v), dev(d_o)
+    o, lse = vt.vt_attn_fwd(tq, tk, tv, causal, cfg.scale)
+    grads = [torch.full_like(t, float("nan")) for t in (tq, tk, tv)]
+    vt.vt_attn_bwd(tq, tk, tv, o, tdo, lse, causal, cfg.scale, *grads)
+    torch.cuda.synchronize()
+    assert vt.vt_attn_device_status()[0] == 0
+    for nm, a, b in zip(("dQ", "dK", "dV"), grads, orc.attn_bwd(q, k, v, d_o, causal, cfg.scale)):
+        a = host(a)
+        assert not np.isnan(a).any(), nm
+        assert np.abs(a - b).max() <= TOL_GRAD * np.abs(b).max() + 1e-5, nm
+
+
+@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,D,causal,seed", [c for c in _cases(40, 6, 128) if c[5] > 64][:12])
+def test_random_shapes_single_pass_backward(vt, B, Hq, Hkv, Sq, Sk, D, causal, seed):
+    """The opt-in single-pass backward (fixed-point dQ accumulation) on random shapes with 64 < D <= 128."""
+    import os
+    import torch
+    cfg = AttnConfig("fuzz_fused", seed, B, Hq, Hkv, Sq, Sk, D, causal, True)
+    q, k, v, d_o = make_inputs(cfg)
+    tq, tk, tv, tdo = dev(q), dev(k), dev(v), dev(d_o)
+    o, lse = vt.vt_attn_fwd(tq, tk, tv, causal, cfg.scale)
+    old = os.environ.get("VT_ATTN_BWD_PATH")
+    os.environ["VT_ATTN_BWD_PATH"] = "fused"
+    try:
+        assert vt.vt_attn_bwd_kernel_kind(B, Hq, Hkv, Sq, Sk, D) == 1
+        grads = vt.vt_attn_bwd(tq, tk, tv, o, tdo, lse, causal, cfg.scale)
+    finally:
+        if old is None:
+            os.environ.pop("VT_ATTN_BWD_PATH", None)
+        else:
+            os.environ["VT_ATTN_BWD_PATH"] = old
+    torch.cuda.synchronize()
+    assert vt.vt_attn_device_status()[0] == 0
+    for nm, a, b in zip(("dQ", "dK", "dV"), grads, orc.attn_bwd(q, k, v, d_o, causal, cfg.scale)):
+        a = host(a)
+        assert not np.isnan(a).any(), nm
+        assert np.abs(a - b).max() <= TOL_GRAD * np.abs(b).max() + 1e-5, nm
+
+
 @pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,D,causal,seed", _cases(16, 2, 256))
 def test_random_shapes_forward_wide_heads_and_splitkv(vt, B, Hq, Hkv, Sq, Sk, D, causal, seed):
     import torch
