@@ -304,13 +304,24 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
         float l = 0.0f;
         bool ok = true;
         if (ROPE) {
-            // this thread's query row, in place: chunk c (8 elements) of the first half pairs with chunk c of the second
-            // half; in the 128-byte-swizzled tile the 16-byte chunk j of row r sits at chunk j ^ (r & 7) of that row
-            ok = mbar_wait(q_full, 0, abort_flag, p.guard, status_word(FWD_KERNEL_ID, ROLE_SOFTMAX, 0xFFFF));
-            if (ok && q0 + r < Sq) {
+            // This thread's query row, in place: chunk c (8 elements) of the first half pairs with chunk c of the second
+            // half; in the 128-byte-swizzled tile the 16-byte chunk j of row r sits at chunk j ^ (r & 7) of that row.
+            // The row's cosines and sines (D / 2 of each) are requested BEFORE the wait for the tile, so their latency
+            // overlaps the tile's own load; read-only loads, all in flight at once.
+            const bool have_row = q0 + r < Sq;
+            float4 cs4[D / 8], sn4[D / 8];
+            if (have_row) {
                 const size_t pos = static_cast<size_t>(p.rope_pos0 + q0 + r);
                 const float4 *ct = reinterpret_cast<const float4 *>(p.rope_cos + pos * (D / 2));
                 const float4 *st = reinterpret_cast<const float4 *>(p.rope_sin + pos * (D / 2));
+#pragma unroll
+                for (int i = 0; i < D / 8; ++i) {
+                    cs4[i] = __ldg(ct + i);
+                    sn4[i] = __ldg(st + i);
+                }
+            }
+            ok = mbar_wait(q_full, 0, abort_flag, p.guard, status_word(FWD_KERNEL_ID, ROLE_SOFTMAX, 0xFFFF));
+            if (ok && have_row) {
                 uint8_t *rowp = sQ + r * 128;
 #pragma unroll
                 for (int ch = 0; ch < D / 16; ++ch) {
@@ -318,7 +329,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant_
                     uint4 *pb = (D == 128) ? reinterpret_cast<uint4 *>(rowp + QBOX_BYTES + ((ch ^ (r & 7)) << 4))
                                            : reinterpret_cast<uint4 *>(rowp + (((ch + 4) ^ (r & 7)) << 4));
                     const uint4 a = *pa, bq = *pb;
-                    const float4 c0 = ct[2 * ch], c1 = ct[2 * ch + 1], s0 = st[2 * ch], s1 = st[2 * ch + 1];
+                    const float4 c0 = cs4[2 * ch], c1 = cs4[2 * ch + 1], s0 = sn4[2 * ch], s1 = sn4[2 * ch + 1];
                     const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
                     const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
                     const uint32_t aw[4] = {a.x, a.y, a.z, a.w}, bw[4] = {bq.x, bq.y, bq.z, bq.w};

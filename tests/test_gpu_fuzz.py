@@ -1,6 +1,8 @@
 """Seeded random shapes through the forward and backward entry points against the fp64 oracle: batch, heads, group size,
 both sequence lengths (from a single row up to several tiles with ragged tails), every head dimension the library takes
 and all three mask modes, in combinations nobody wrote down by hand."""
+import os
+
 import numpy as np
 import pytest
 
@@ -9,6 +11,31 @@ from oracle import attn_oracle as orc
 from paper_2601_16238_b200.inputs import AttnConfig, make_inputs
 
 pytestmark = pytest.mark.gpu
+
+# VT_FUZZ_SCALE=k multiplies the number of random cases of every test in this file (default 1: what a normal test run
+# does; the tolerance floors quoted in the design notes come from a run with 70, about 2 500 batched and 1 100 packed cases)
+SCALE = max(1, int(os.environ.get("VT_FUZZ_SCALE", "1")))
+
+
+def zero_floor(n_terms):
+    """Absolute slack for gradients that are exactly zero in exact arithmetic (a single visible key: P = 1, dS = 0, so dQ
+    and dK vanish): the kernel's dS is then the fp32 rounding of <dO, v> - <dO, o> (~1e-6 of either for N(0,1) data),
+    and a gradient sums n_terms of them with random signs."""
+    return max(1e-5, 2e-6 * float(np.sqrt(n_terms)))
+
+
+def grad_tol(nm, ref, q, k, d_o, o, scale, rows, keys):
+    """Tolerance for one gradient: the relative bound on its largest element, the floor for exactly-zero gradients, and,
+    for dQ and dK, what the bf16 rounding of O costs.  The backward's row term delta_i = <dO_i, O_i> reads the rounded
+    output, so it is off by up to 2^-9 sum_d |dO_id O_id|; with one or two visible keys dP - delta cancels almost
+    completely, the gradient itself is small, and that error is no longer small beside it.  It reaches dQ_i through
+    scale * sum_j P_ij K_j (weights summing to 1) and dK_j through scale * sum_i P_ij Q_i (random signs over the rows)."""
+    tol = TOL_GRAD * np.abs(ref).max() + zero_floor(max(rows, keys))
+    if nm != "dV":
+        d_delta = 2.0 ** -9 * np.abs(d_o.astype(np.float64) * o.astype(np.float64)).sum(-1).max()
+        other = np.abs(k).max() if nm == "dQ" else np.abs(q).max() * np.sqrt(rows)
+        tol += scale * d_delta * float(other)
+    return tol
 
 
 def _cases(n, seed, max_d):
@@ -24,7 +51,7 @@ def _cases(n, seed, max_d):
     return out
 
 
-@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,D,causal,seed", _cases(36, 1, 128))
+@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,D,causal,seed", _cases(36 * SCALE, 1, 128))
 def test_random_shapes_forward_and_backward(vt, B, Hq, Hkv, Sq, Sk, D, causal, seed):
     import torch
     cfg = AttnConfig("fuzz", seed, B, Hq, Hkv, Sq, Sk, D, causal, True)
@@ -48,14 +75,14 @@ def test_random_shapes_forward_and_backward(vt, B, Hq, Hkv, Sq, Sk, D, causal, s
     for nm, a, b in zip(("dQ", "dK", "dV"), grads, orc.attn_bwd(q, k, v, d_o, causal, cfg.scale)):
         a = host(a)
         assert not np.isnan(a).any(), nm
-        assert np.abs(a - b).max() <= TOL_GRAD * np.abs(b).max() + 1e-5, nm
+        assert np.abs(a - b).max() <= grad_tol(nm, b, q, k, d_o, o_h, cfg.scale, Sq * (Hq // Hkv), Sk), nm
 
 
 def _wide_cases(n, seed):
     return [c[:5] + (136 + 8 * (c[7] * 7 % 16),) + c[6:] for c in _cases(n, seed, 128)]      # D in 136 .. 256
 
 
-@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,D,causal,seed", _wide_cases(16, 5))
+@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,D,causal,seed", _wide_cases(16 * SCALE, 5))
 def test_random_shapes_backward_above_128_columns(vt, B, Hq, Hkv, Sq, Sk, D, causal, seed):
     import torch
     cfg = AttnConfig("fuzz_wide", seed, B, Hq, Hkv, Sq, Sk, D, causal, True)
@@ -66,13 +93,14 @@ def test_random_shapes_backward_above_128_columns(vt, B, Hq, Hkv, Sq, Sk, D, cau
     vt.vt_attn_bwd(tq, tk, tv, o, tdo, lse, causal, cfg.scale, *grads)
     torch.cuda.synchronize()
     assert vt.vt_attn_device_status()[0] == 0
+    o_h = host(o)
     for nm, a, b in zip(("dQ", "dK", "dV"), grads, orc.attn_bwd(q, k, v, d_o, causal, cfg.scale)):
         a = host(a)
         assert not np.isnan(a).any(), nm
-        assert np.abs(a - b).max() <= TOL_GRAD * np.abs(b).max() + 1e-5, nm
+        assert np.abs(a - b).max() <= grad_tol(nm, b, q, k, d_o, o_h, cfg.scale, Sq * (Hq // Hkv), Sk), nm
 
 
-@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,D,causal,seed", [c for c in _cases(40, 6, 128) if c[5] > 64][:12])
+@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,D,causal,seed", [c for c in _cases(40 * SCALE, 6, 128) if c[5] > 64][:12 * SCALE])
 def test_random_shapes_single_pass_backward(vt, B, Hq, Hkv, Sq, Sk, D, causal, seed):
     """The opt-in single-pass backward (fixed-point dQ accumulation) on random shapes with 64 < D <= 128."""
     import os
@@ -93,13 +121,14 @@ def test_random_shapes_single_pass_backward(vt, B, Hq, Hkv, Sq, Sk, D, causal, s
             os.environ["VT_ATTN_BWD_PATH"] = old
     torch.cuda.synchronize()
     assert vt.vt_attn_device_status()[0] == 0
+    o_h = host(o)
     for nm, a, b in zip(("dQ", "dK", "dV"), grads, orc.attn_bwd(q, k, v, d_o, causal, cfg.scale)):
         a = host(a)
         assert not np.isnan(a).any(), nm
-        assert np.abs(a - b).max() <= TOL_GRAD * np.abs(b).max() + 1e-5, nm
+        assert np.abs(a - b).max() <= grad_tol(nm, b, q, k, d_o, o_h, cfg.scale, Sq * (Hq // Hkv), Sk), nm
 
 
-@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,D,causal,seed", _cases(16, 2, 256))
+@pytest.mark.parametrize("B,Hq,Hkv,Sq,Sk,D,causal,seed", _cases(16 * SCALE, 2, 256))
 def test_random_shapes_forward_wide_heads_and_splitkv(vt, B, Hq, Hkv, Sq, Sk, D, causal, seed):
     import torch
     cfg = AttnConfig("fuzz", seed, B, Hq, Hkv, Sq, Sk, D, causal, False)
@@ -135,7 +164,7 @@ def _packed_cases(n, seed):
     return out
 
 
-@pytest.mark.parametrize("Hq,Hkv,D,causal,lens_q,lens_k,seed", _packed_cases(16, 3))
+@pytest.mark.parametrize("Hq,Hkv,D,causal,lens_q,lens_k,seed", _packed_cases(16 * SCALE, 3))
 def test_random_packed_batches(vt, Hq, Hkv, D, causal, lens_q, lens_k, seed):
     import torch
     from paper_2601_16238_b200.inputs import normal_bf16
@@ -162,10 +191,10 @@ def test_random_packed_batches(vt, Hq, Hkv, D, causal, lens_q, lens_k, seed):
     for nm, a, b in zip(("dQ", "dK", "dV"), grads, orc.attn_bwd_varlen(q, k, v, d_o, cu_q, cu_k, causal, scale)):
         a = host(a)
         assert not np.isnan(a).any(), nm
-        assert np.abs(a - b).max() <= TOL_GRAD * np.abs(b).max() + 1e-5, nm
+        assert np.abs(a - b).max() <= grad_tol(nm, b, q, k, d_o, o_h, scale, max(lens_q) * (Hq // Hkv), max(lens_k)), nm
 
 
-@pytest.mark.parametrize("Hq,Hkv,D,causal,lens_q,lens_k,seed", _packed_cases(12, 4))
+@pytest.mark.parametrize("Hq,Hkv,D,causal,lens_q,lens_k,seed", _packed_cases(12 * SCALE, 4))
 def test_random_packed_batches_splitkv(vt, Hq, Hkv, D, causal, lens_q, lens_k, seed):
     import torch
     from paper_2601_16238_b200.inputs import normal_bf16
