@@ -479,6 +479,8 @@ int vt_attn_fwd_bwd_host_f16(const void *q_host, const void *k_host, const void 
  * device, clears it if set (waiting once more), and returns VT_ATTN_OK or
  * VT_ATTN_ERR_DEVICE_TIMEOUT.  detail (host, may be NULL) receives the raw word: bits
  * 0-7 kernel id, 8-15 waiting role, 16-31 tile index.  Not for use during stream capture.
+ * Kernel ids: 1 one-tile forward, 2 dK/dV, 3 dQ, 4 two-tile forward, 5 forward with two tiles
+ * in sequence, 6 / 7 dK/dV and dQ above 128 columns, 8 single-pass backward, 9 self-test.
  *
  * vt_attn_device_status_async and vt_attn_device_status_clear are the non-blocking
  * pieces for callers that own their synchronisation points: the first enqueues a copy

@@ -36,7 +36,7 @@ constexpr int FUSED_THREADS = 512;
 #define VT_FUSED_DRAIN_REGS 144
 #define VT_FUSED_PRODUCER_REGS 104
 #endif
-constexpr uint32_t FUSED_KERNEL_ID = 4;
+constexpr uint32_t FUSED_KERNEL_ID = 8;
 constexpr int DQ_FIXED_BITS = 28;              // |contribution sums| * scale < 2^29 (see dq_fixed_scale)
 
 // Power of two that maps the bound R (|dQ column sums| <= R before the softmax scale) to < 2^28; 1 when R is 0 or not finite.

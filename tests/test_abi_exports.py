@@ -176,6 +176,19 @@ def test_product_path_does_not_import_the_oracle():
                 assert "oracle" not in text.lower() or f == "inputs.py", f"{f} mentions the oracle"
 
 
+def test_status_word_kernel_ids_are_distinct():
+    """A timed-out wait names its kernel in the low byte of the status word: two kernels must not share an id."""
+    import re
+    ids = {}
+    csrc = os.path.join(ROOT, "paper_2601_16238_b200", "csrc")
+    for f in sorted(os.listdir(csrc)):
+        for name, val in re.findall(r"constexpr uint32_t (\w+_KERNEL_ID) = (\d+);", open(os.path.join(csrc, f)).read()):
+            assert int(val) not in ids, f"{name} and {ids[int(val)]} share id {val}"
+            assert 0 < int(val) < 256
+            ids[int(val)] = name
+    assert len(ids) >= 9
+
+
 def test_splitkv_plan_and_workspace(lib):
     # decoding: 4 query heads per KV head, one query each -> the group shares a tile; 512 steps of 64 keys
     used, share = vt.vt_attn_fwd_splitkv_plan(4, 32, 8, 1, 32768, 128, 0)
