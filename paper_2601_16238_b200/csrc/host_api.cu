@@ -21,11 +21,11 @@ struct Chunk {
 
 // Chunks of about equal size: whole batches when there are at least as many batches as chunks, else KV-head ranges inside
 // each batch.  `min_units` keeps a chunk large enough to fill the GPU (units = (batch, KV head) groups).
-static int make_chunks(int B, int Hkv, int min_units, Chunk (&out)[MAX_CHUNKS * 2])
+static int make_chunks(int B, int Hkv, int min_units, int max_chunks, Chunk (&out)[MAX_CHUNKS * 2])
 {
     const int units = B * Hkv;
     int want = units / (min_units > 0 ? min_units : 1);
-    if (want > MAX_CHUNKS) want = MAX_CHUNKS;
+    if (want > max_chunks) want = max_chunks;
     if (want < 1) want = 1;
     int n = 0;
     if (want <= B) {
@@ -129,9 +129,16 @@ static int run_chunked(bool f16, const HostArgs &h, int B, int Hq, int Hkv, int 
     // a chunk should still fill the GPU: its smallest grid (one block per 128-key tile and KV head in the backward, one block
     // per SM; per query tile or pair of tiles and query head in the forward, two per SM) gets at least one wave
     const long long per_unit = with_backward ? (Sk + TILE - 1) / TILE : static_cast<long long>((Sq + 2 * TILE - 1) / (2 * TILE)) * G;
-    const int min_units = static_cast<int>(((with_backward ? NUM_SMS : 2 * NUM_SMS) + per_unit - 1) / per_unit);
+    int min_units = static_cast<int>(((with_backward ? NUM_SMS : 2 * NUM_SMS) + per_unit - 1) / per_unit);
+    // When the copies take much longer than the kernels (a forward over PCIe: ~50 GB/s in against ~800 TFLOP/s), what the
+    // call costs beyond its input copies is the LAST chunk's kernel and output copy: smaller chunks (a quarter of a wave is
+    // enough, the kernels are not what is waited for) and twice as many of them shorten that tail.
+    const double in_bytes = (with_backward ? 2.0 : 1.0) * static_cast<double>(s.q_bytes) + 2.0 * static_cast<double>(s.kv_bytes);
+    const double flops = 4.0 * B * Hq * static_cast<double>(Sq) * Sk * D * (causal ? 0.5 : 1.0) * (with_backward ? 3.5 : 1.0);
+    const bool copy_bound = 2.0 * flops / 800e12 < in_bytes / 50e9;
+    if (copy_bound) min_units = (min_units + 3) / 4;
     Chunk chunks[MAX_CHUNKS * 2];
-    const int n = make_chunks(B, Hkv, min_units, chunks);
+    const int n = make_chunks(B, Hkv, min_units, copy_bound ? 2 * MAX_CHUNKS : MAX_CHUNKS, chunks);
     SideStreams *ss = nullptr;
     int rc = side_streams(&ss);
     if (rc != VT_ATTN_OK) return rc;

@@ -89,10 +89,9 @@ def test_host_buffer_entry_points_match_device_path(vt):
 
 def test_host_buffer_entry_points_with_several_chunks(vt):
     """A problem large enough for the host entry points to cut it into chunks that alternate between two streams (whole
-    batches in the forward call, KV-head ranges inside each batch in the forward + backward call); GQA so that a chunk's
-    query heads are a multiple of its KV heads.  The chunks of the forward call get the same kernel as the whole problem,
-    so its result is the same bits; the chunks of the forward + backward call are smaller and may get the other forward
-    kernel, so that one is compared within rounding."""
+    batches or KV-head ranges inside each batch, more and smaller ones when the copies outweigh the kernels); GQA so that
+    a chunk's query heads are a multiple of its KV heads.  A chunk may get another forward kernel than the whole problem
+    (fewer heads per launch), so the results are compared within rounding, not bit for bit."""
     import torch
     B, Hq, Hkv, S, D = 4, 16, 8, 4096, 128
     gen = torch.Generator(device="cuda").manual_seed(99)
@@ -106,7 +105,9 @@ def test_host_buffer_entry_points_with_several_chunks(vt):
     vt.vt_attn_fwd_host(hq, hk, hv, ho, hlse, False, scale, st)
     o, lse = vt.vt_attn_fwd(q, k, v, False, scale)
     torch.cuda.synchronize()
-    assert torch.equal(ho, o.cpu()) and torch.equal(hlse, lse.cpu())
+    assert vt.vt_attn_device_status()[0] == 0
+    assert (hlse - lse.cpu()).abs().max() <= 1e-4
+    assert (ho.float() - o.cpu().float()).abs().max() <= 2.0 ** -6 * o.float().abs().max().item()
     hdq = torch.empty_like(hq).pin_memory(); hdk = torch.empty_like(hk).pin_memory(); hdv = torch.empty_like(hv).pin_memory()
     st2 = torch.empty(vt.vt_attn_host_staging_bytes(*dims, True), dtype=torch.uint8, device="cuda")
     vt.vt_attn_fwd_bwd_host(hq, hk, hv, hdo, ho, hlse, hdq, hdk, hdv, True, scale, st2)
