@@ -62,6 +62,10 @@ NCU_TRAFFIC_BYTES = {
     # (Delta 273.9 + dK/dV 397.4 + dQ 454.0 MB)
     "gqa_long": 312.3e6,
     "gqa_long_bwd": 1125.3e6,
+    # profiles/attn_fwd_kernel_d64_s4096_nc.md: 101.1 MB read + 17.3 MB written (part of O still in L2 at the end)
+    "d64_s4096_nc": 118.4e6,
+    # profiles/fwd_bwd_kernels_d256_s4096_nc.md: forward 201.5 MB read + 48.0 MB written
+    "d256_s4096_nc": 249.5e6,
 }
 NCU_TRAFFIC_NOTE = {}
 

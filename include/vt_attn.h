@@ -57,7 +57,7 @@ extern "C" {
 
 #define VT_ATTN_OK 0
 #define VT_ATTN_ERR_INVALID_ARGUMENT (-1)    /* null/misaligned pointer, bad shape or scale */
-#define VT_ATTN_ERR_UNSUPPORTED (-2)         /* head dim not a multiple of 8 in [8,256] ([8,128] in the packed and host-buffer entry points); device is not sm_100 */
+#define VT_ATTN_ERR_UNSUPPORTED (-2)         /* head dim not a multiple of 8 in [8,256] ([8,128] in the packed entry points); device is not sm_100 */
 #define VT_ATTN_ERR_WORKSPACE_TOO_SMALL (-3) /* workspace_bytes below vt_attn_bwd_workspace_bytes */
 #define VT_ATTN_ERR_CUDA (-4)                /* a CUDA runtime / driver call failed */
 #define VT_ATTN_ERR_DEVICE_TIMEOUT (-5)      /* reported by vt_attn_device_status only */

@@ -197,7 +197,7 @@ static int run_chunked(bool f16, const HostArgs &h, int B, int Hq, int Hkv, int 
 extern "C" size_t vt_attn_host_staging_bytes(int B, int Hq, int Hkv, int Sq, int Sk, int D, int with_backward)
 {
     vt::Shape s{B, Hq, Hkv, Sq, Sk, D};
-    if (vt::check_shape(s, 1.0f) != VT_ATTN_OK) return 0;
+    if (vt::check_shape(s, 1.0f, vt::MAX_HEAD_DIM_FWD) != VT_ATTN_OK) return 0;
     return vt::plan(B, Hq, Hkv, Sq, Sk, D, with_backward != 0).total;
 }
 
@@ -207,7 +207,7 @@ static int fwd_host_entry(bool f16, const void *q_host, const void *k_host, cons
 {
     using namespace vt;
     Shape sh{B, Hq, Hkv, Sq, Sk, D};
-    int rc = check_shape(sh, scale);
+    int rc = check_shape(sh, scale, MAX_HEAD_DIM_FWD);
     if (rc != VT_ATTN_OK) return rc;
     if (!q_host || !k_host || !v_host || !o_host || !lse_host || !ptr_ok(staging, 256)) return VT_ATTN_ERR_INVALID_ARGUMENT;
     if (causal < 0 || causal > 2) return VT_ATTN_ERR_INVALID_ARGUMENT;
@@ -240,7 +240,7 @@ static int fwd_bwd_host_entry(bool f16, const void *q_host, const void *k_host, 
 {
     using namespace vt;
     Shape sh{B, Hq, Hkv, Sq, Sk, D};
-    int rc = check_shape(sh, scale);
+    int rc = check_shape(sh, scale, MAX_HEAD_DIM_FWD);
     if (rc != VT_ATTN_OK) return rc;
     if (!q_host || !k_host || !v_host || !d_o_host || !o_host || !lse_host || !dq_host || !dk_host || !dv_host ||
         !ptr_ok(staging, 256))

@@ -151,11 +151,14 @@ def test_argument_validation_returns_before_any_cuda_call(lib):
     assert lib.vt_attn_fwd_host(*([_fake()] * 5), 1, 2, 2, 128, 128, 64, 0, 0.125, _fake(0x10000), 16, None) \
         == vt.ERR_WORKSPACE_TOO_SMALL
     assert lib.vt_attn_selftest_timeout(0, None) == vt.ERR_INVALID_ARGUMENT
-    # head dimensions above 128 exist only in the [B, H, S, D] forward and backward entry points: the packed ones and the host-buffer
-    # ones answer "unsupported", as does a V width outside [8, 256]
+    # head dimensions above 128 exist only in the [B, H, S, D] forward and backward entry points and the host-buffer ones
+    # built on them: the packed ones answer "unsupported", as does a V width outside [8, 256]
     cu = _fake(0x2000)
     assert lib.vt_attn_fwd_varlen(*([_fake()] * 5), cu, cu, 2, 2, 2, 256, 256, 128, 128, 192, 0, 0.1, None) == vt.ERR_UNSUPPORTED
-    assert lib.vt_attn_fwd_host(*([_fake()] * 5), 1, 2, 2, 128, 128, 192, 0, 0.125, _fake(0x10000), 1 << 30, None) == vt.ERR_UNSUPPORTED
+    assert lib.vt_attn_fwd_host(*([_fake()] * 5), 1, 2, 2, 128, 128, 192, 0, 0.125, _fake(0x10000), 16, None) == vt.ERR_WORKSPACE_TOO_SMALL
+    assert lib.vt_attn_fwd_host(*([_fake()] * 5), 1, 2, 2, 128, 128, 264, 0, 0.125, _fake(0x10000), 1 << 30, None) == vt.ERR_UNSUPPORTED
+    assert vt.vt_attn_host_staging_bytes(1, 2, 2, 128, 128, 256, True) > vt.vt_attn_host_staging_bytes(1, 2, 2, 128, 128, 256, False) > 0
+    assert vt.vt_attn_host_staging_bytes(1, 2, 2, 128, 128, 264, False) == 0
     assert lib.vt_attn_fwd_dv(*([_fake()] * 5), 1, 2, 2, 128, 128, 192, 264, 0, 0.125, None) == vt.ERR_UNSUPPORTED
     assert lib.vt_attn_fwd_dv(*([_fake()] * 5), 1, 2, 2, 128, 128, 192, 100, 0, 0.125, None) == vt.ERR_UNSUPPORTED
 

@@ -251,10 +251,12 @@ def test_forward_with_its_own_v_width(vt, B, Hq, Hkv, Sq, Sk, D, Dv, causal):
         assert torch.equal(o1, o) and torch.equal(lse1, lse)
 
 
-def test_host_buffer_entry_points_with_another_head_dim(vt):
-    """The host-buffer entry points stage rows of the real length (D = 96: 192-byte rows) and give the bits of the device path."""
+@pytest.mark.parametrize("D", [96, 192, 256])
+def test_host_buffer_entry_points_with_another_head_dim(vt, D):
+    """The host-buffer entry points stage rows of the real length (D = 96: 192-byte rows) and give the bits of the device
+    path, also above 128 columns (the backward in two column halves)."""
     import torch
-    cfg = AttnConfig("hd_host", 25, 3, 4, 2, 300, 300, 96, 1, True)
+    cfg = AttnConfig("hd_host", 25, 3, 4, 2, 300, 300, D, 1, True)
     bits = make_inputs(cfg)
     hq, hk, hv, hdo = (torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory() for x in bits)
     ho = torch.empty_like(hq).pin_memory(); hlse = torch.empty(hq.shape[:3], dtype=torch.float32).pin_memory()
