@@ -21,6 +21,8 @@ SHAPES = [
     (1, 2, 2, 450, 190, 200, 2),          # fewer keys than queries: leading rows see nothing
     (1, 3, 3, 1, 1, 256, 1),
     (1, 2, 2, 640, 640, 256, 1),
+    (1, 2, 1, 4096, 4096, 256, 0),        # two full-length heads of the benchmark's d256_s4096_nc workload (one KV head)
+    (1, 2, 2, 2048, 2048, 256, 1),
 ]
 
 
