@@ -227,7 +227,7 @@ int vt_attn_fwd_varlen(const void *q, const void *k, const void *v, void *o, flo
  * vt_attn_fwd with V (and O) of their own head dimension Dv, e.g. Q, K of 192 columns against V of
  * 128: q [B, Hq, Sq, D], k [B, Hkv, Sk, D], v [B, Hkv, Sk, Dv], o [B, Hq, Sq, Dv], bfloat16;
  * D and Dv multiples of 8 in [8, 256].  Runs in the kernel built for the larger of the two (rounded
- * up to 64, 128 or 256 columns).  Forward only.
+ * up to 64, 128 or 256 columns).  Its backward is vt_attn_bwd_dv.
  */
 int vt_attn_fwd_dv(const void *q, const void *k, const void *v, void *o, float *lse,
                    int B, int Hq, int Hkv, int Sq, int Sk, int D, int Dv,
