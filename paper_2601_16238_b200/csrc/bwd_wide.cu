@@ -4,11 +4,11 @@
 // accumulators in tensor memory; at 256 columns neither fits.  Here the stationary side stays 128 rows (at 256 columns:
 // 64 KB per tile) and the streamed side is cut to 64 rows, so every score tile is 128 x 64:
 //
-//   bwd_dkdv_wide_kernel : one block per (batch, KV head, 128-key tile, column half).  K and V (all 256 columns) stay in
-//       shared memory; the query heads of the group are walked 64 queries at a time (Q in two slots, dO in one).
-//       S^T = K Q^T and dP^T = V dO^T contract over all columns; dV and dK are accumulated for ONE half of the
-//       columns per block (two accumulators of 128 columns next to S^T and dP^T in tensor memory), so the grid's
-//       second dimension runs the walk twice - the price of 512 tensor-memory columns.
+//   bwd_dkdv_wide_kernel : two blocks per (batch, KV head, 128-key tile), one per output tensor (dK and dV of 256
+//       columns together would fill tensor memory).  K stays in shared memory; the query heads of the group are walked
+//       64 queries at a time (Q in two slots) and S^T = K Q^T contracts over all columns in both blocks.  The dK block also
+//       holds V, forms dP^T = V dO^T and dS^T and accumulates dK += dS^T Q (N = 256); the dV block only needs P^T and
+//       accumulates dV += P^T dO, with two score buffers and two dO slots.
 //   bwd_dq_wide_kernel   : one block per (batch, query head, 128-query tile).  Q and dO stay in shared memory, K (two
 //       slots) and V (one slot) stream by in tiles of 64 keys; dQ (256 columns) is accumulated in tensor memory.
 //
@@ -41,11 +41,13 @@ struct DkdvWideSmem {
     static constexpr int OFF_ROWS = OFF_DO + TILE64_BYTES;           // [slot][-lse2 64 | -delta 64]
     static constexpr int OFF_BAR = OFF_ROWS + ROW_SLOTS * 2 * WIDE_N * 4;
     static constexpr int BYTES = OFF_BAR + 256;                      // no alignment slack: the kernel checks the base address
-    // TMEM columns: S^T [0,64) (P^T, bf16, over its first 32), dP^T [64,128) (dS^T over its first 32), dV half [128,256),
-    // dK half [256,384)
+    // TMEM columns.  dK block: S^T [0,64), dP^T [64,128) (dS^T, 16-bit, over its first 32), dK [128,384).
+    // dV block: two S^T buffers [0,64), [64,128) (P^T, 16-bit, over the first 32 of each), dV [128,384).
     static constexpr int TMEM_COLS = 512;
 };
 
+// grid.y = 0: the block accumulates dK of its key tile (all columns), grid.y = 1: dV.  Both walk the same queries and form
+// the same scores; only the dK block needs dP and dS, only the dV block hands P to the tensor core.
 template <bool CAUSAL, bool F16>
 __global__ void __launch_bounds__(WIDE_THREADS, 1)
 bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
@@ -63,17 +65,21 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem + L::OFF_BAR);
     uint64_t *kv_full = bars + 0;
     uint64_t *final_bar = bars + 1;
-    uint64_t *s_full = bars + 2;
-    uint64_t *dp_full = bars + 3;
-    uint64_t *p_ready = bars + 4;             // 128 arrivals
-    uint64_t *ds_ready = bars + 5;            // 128 arrivals
-    uint64_t *q_full = bars + 6;              // [2]
-    uint64_t *q_empty = bars + 8;             // [2]
-    uint64_t *do_full = bars + 10;
-    uint64_t *do_empty = bars + 11;
-    uint64_t *rows_full = bars + 12;          // [RS] 32 arrivals
-    uint64_t *rows_empty = bars + 12 + RS;    // [RS] one arrival per compute warp
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 12 + 2 * RS);
+    uint64_t *s_full = bars + 2;              // [2] (the dK block uses the first only)
+    uint64_t *dp_full = bars + 4;
+    // 128 arrivals each.  dK block: p_ready[0] = the scores have been read, ds_ready = dS^T is in tensor memory.  dV block:
+    // p_ready[buf] = P^T is in score buffer buf - one barrier per buffer, because with the scores two iterations ahead
+    // the compute warps may finish two iterations before the MMA warp looks, and a single barrier would then have gone
+    // through two phases (the parity the MMA warp waits for would read as "not yet")
+    uint64_t *p_ready = bars + 5;             // [2]
+    uint64_t *ds_ready = bars + 7;
+    uint64_t *q_full = bars + 8;              // [2]
+    uint64_t *q_empty = bars + 10;            // [2]
+    uint64_t *do_full = bars + 12;            // [2] (the dK block uses the first only)
+    uint64_t *do_empty = bars + 14;           // [2]
+    uint64_t *rows_full = bars + 16;          // [RS] 32 arrivals
+    uint64_t *rows_empty = bars + 16 + RS;    // [RS] one arrival per compute warp
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 16 + 2 * RS);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5;
@@ -83,7 +89,7 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         return;
     }
 
-    const int half = blockIdx.y;                          // which 128 columns of dK / dV this block accumulates
+    const bool is_dv = blockIdx.y != 0;                   // block-uniform: the longer dK blocks come first in the launch
     const int bh_kv = blockIdx.x / p.n_tiles;
     const int kt = blockIdx.x % p.n_tiles;
     const int b = bh_kv / p.Hkv;
@@ -96,24 +102,27 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const int n_qi = n_qt - qt_start;
     const int n_it = n_qi * p.G;
     const int dv_w = p.d_v > 0 ? p.d_v : p.d;             // width of V, dO, dV (Q, K, dK: p.d)
-    const int cols_k = min(TILE, p.d - half * TILE);      // real columns of dK in this half (<= 0: none)
-    const int cols_v = min(TILE, dv_w - half * TILE);     // of dV
+    const int out_w = is_dv ? dv_w : p.d;                 // columns of this block's output tensor
     const int kd = (p.d + 15) >> 4;                       // 16-column contraction steps of S^T = K Q^T that hold data
     const int kdv = (dv_w + 15) >> 4;                     // of dP^T = V dO^T
 
     if (threadIdx.x == 0) {
         mbar_init(kv_full, 1);
         mbar_init(final_bar, 1);
-        mbar_init(s_full, 1);
+        mbar_init(&s_full[0], 1);
+        mbar_init(&s_full[1], 1);
         mbar_init(dp_full, 1);
-        mbar_init(p_ready, 128);
+        mbar_init(&p_ready[0], 128);
+        mbar_init(&p_ready[1], 128);
         mbar_init(ds_ready, 128);
         for (int s = 0; s < 2; ++s) {
             mbar_init(&q_full[s], 1);
             mbar_init(&q_empty[s], 1);
         }
-        mbar_init(do_full, 1);
-        mbar_init(do_empty, 1);
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(&do_full[s], 1);
+            mbar_init(&do_empty[s], 1);
+        }
         for (int s = 0; s < RS; ++s) {
             mbar_init(&rows_full[s], 32);
             mbar_init(&rows_empty[s], 4);
@@ -122,11 +131,11 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         fence_mbar_init();
         prefetch_tensormap(&tm_q);
         prefetch_tensormap(&tm_k);
-        prefetch_tensormap(&tm_v);
-        mbar_arrive_expect_tx(kv_full, 2 * TILE128_BYTES);
+        if (!is_dv) prefetch_tensormap(&tm_v);
+        mbar_arrive_expect_tx(kv_full, (is_dv ? 1 : 2) * TILE128_BYTES);       // the dV block never reads V
         for (int kb = 0; kb < WIDE_BOXES; ++kb) {
             tma_load_3d(sK + kb * BOX128_BYTES, &tm_k, kv_full, kb * BOX_COLS, k0, bh_kv);
-            tma_load_3d(sV + kb * BOX128_BYTES, &tm_v, kv_full, kb * BOX_COLS, k0, bh_kv);
+            if (!is_dv) tma_load_3d(sV + kb * BOX128_BYTES, &tm_v, kv_full, kb * BOX_COLS, k0, bh_kv);
         }
         if (n_it > 0) {
             mbar_arrive_expect_tx(&q_full[0], TILE64_BYTES);
@@ -156,15 +165,19 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             }
         }
     } else if (warp == 2) {
-        if (lane == 0) {                           // dO tiles: one slot, reloaded as soon as dV of the iteration has completed
+        if (lane == 0) {
+            // dO tiles.  dK block: one slot, reloaded as soon as dP of the iteration has completed.  dV block: two slots (the
+            // second in the memory the V tile would take), since dV(i + 1) follows dV(i) within a few hundred cycles.
             prefetch_tensormap(&tm_do);
             for (int it = 0; it < n_it; ++it) {
                 const int hq = hkv * p.G + it / n_qi;
                 const int q0 = (qt_start + it % n_qi) * WIDE_N;
-                if (!mbar_wait(do_empty, (it & 1) ^ 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_LOAD, it))) break;
-                mbar_arrive_expect_tx(do_full, TILE64_BYTES);
+                const int sl = is_dv ? (it & 1) : 0;
+                uint8_t *dst = sl ? sV : sdO;
+                if (!mbar_wait(&do_empty[sl], ((is_dv ? (it >> 1) : it) & 1) ^ 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_LOAD, it))) break;
+                mbar_arrive_expect_tx(&do_full[sl], TILE64_BYTES);
                 for (int kb = 0; kb < WIDE_BOXES; ++kb)
-                    tma_load_3d(sdO + kb * BOX64_BYTES, &tm_do, do_full, kb * BOX_COLS, q0, b * p.Hq + hq);
+                    tma_load_3d(dst + kb * BOX64_BYTES, &tm_do, &do_full[sl], kb * BOX_COLS, q0, b * p.Hq + hq);
             }
         }
     } else if (warp == 3) {
@@ -190,16 +203,14 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             mbar_arrive(&rows_full[sl]);
         }
     } else if (warp == 1) {
-        // MMA issuer.  Per iteration: dV(i), S(i+1), dK(i), dP(i+1) - the order of the 128-column kernel.
+        // MMA issuer
         constexpr uint32_t IDESC_S = make_idesc(128, WIDE_N, fmt16<F16>(), fmt16<F16>(), 0, 0);
-        const uint32_t IDESC_GV = make_idesc(128, ((max(cols_v, 8) + 15) >> 4) * 16, fmt16<F16>(), fmt16<F16>(), 0, 1);
-        const uint32_t IDESC_GK = make_idesc(128, ((max(cols_k, 8) + 15) >> 4) * 16, fmt16<F16>(), fmt16<F16>(), 0, 1);
+        const uint32_t IDESC_G = make_idesc(128, ((out_w + 15) >> 4) * 16, fmt16<F16>(), fmt16<F16>(), 0, 1);
         const uint32_t tmem_u = __shfl_sync(0xFFFFFFFFu, tmem_base, 0);
         const uint64_t dK0 = smem_desc_sw128(smem_u32(sK), 16, 1024), dV0 = smem_desc_sw128(smem_u32(sV), 16, 1024);
-        // dO and Q as MN-major B operands restricted to this block's column half: boxes 2 * half and 2 * half + 1
-        const uint64_t dDOm = smem_desc_sw128(smem_u32(sdO + half * 2 * BOX64_BYTES), BOX64_BYTES, 1024);
         bool ok = mbar_wait(kv_full, 0, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, 0xFFFF));
-        auto issue_s = [&](int it) -> bool {       // S^T = K Q^T over all columns
+        // S^T = K Q^T over all columns into score buffer `buf`; free_q: nothing else reads this Q tile (dV block)
+        auto issue_s = [&](int it, int buf, bool free_q) -> bool {
             const int sl = it & 1;
             if (!mbar_wait(&q_full[sl], (it >> 1) & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it))) return false;
             tc_fence_after_sync();
@@ -208,63 +219,79 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
                 for (int k = 0; k < WIDE_D / 16; ++k)
                     if (k < kd)
-                        umma_ss(tmem_u, desc_advance(dK0, (k / 4) * BOX128_BYTES + (k % 4) * 32),
+                        umma_ss(tmem_u + buf * WIDE_N, desc_advance(dK0, (k / 4) * BOX128_BYTES + (k % 4) * 32),
                                 desc_advance(dQs, (k / 4) * BOX64_BYTES + (k % 4) * 32), IDESC_S, k > 0 ? 1u : 0u);
-                umma_commit(s_full);
+                umma_commit(&s_full[buf]);
+                if (free_q) umma_commit(&q_empty[sl]);
             }
             __syncwarp();
             return true;
         };
-        auto issue_dp = [&](int it) -> bool {      // dP^T = V dO^T over all columns
-            if (!mbar_wait(do_full, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it))) return false;
-            tc_fence_after_sync();
-            if (elect_one()) {
-                const uint64_t dDOs = smem_desc_sw128(smem_u32(sdO), 16, 1024);
-#pragma unroll
-                for (int k = 0; k < WIDE_D / 16; ++k)
-                    if (k < kdv)
-                        umma_ss(tmem_u + 64, desc_advance(dV0, (k / 4) * BOX128_BYTES + (k % 4) * 32),
-                                desc_advance(dDOs, (k / 4) * BOX64_BYTES + (k % 4) * 32), IDESC_S, k > 0 ? 1u : 0u);
-                umma_commit(dp_full);
-            }
-            __syncwarp();
-            return true;
-        };
-        if (ok && n_it > 0) ok = issue_s(0);
-        if (ok && n_it > 0) ok = issue_dp(0);
-        for (int it = 0; it < n_it && ok; ++it) {
-            const int sl = it & 1;
-            ok = mbar_wait(p_ready, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it));
-            if (!ok) break;
-            tc_fence_after_sync();
-            if (elect_one()) {                     // dV[:, half] += P^T dO[:, half]   (16 query rows per instruction)
-                if (cols_v > 0) {
-#pragma unroll
-                    for (int k = 0; k < WIDE_N / 16; ++k)
-                        umma_ts(tmem_u + 128, tmem_u + k * 8, desc_advance(dDOm, k * 2048), IDESC_GV, (it > 0 || k > 0) ? 1u : 0u);
-                }
-                umma_commit(do_empty);
-            }
-            __syncwarp();
-            if (it + 1 < n_it) {
-                ok = issue_s(it + 1);              // overwrites P^T(it): ordered behind dV(it)
+        if (is_dv) {
+            // Per iteration: dV(i), then S(i+2) into the score buffer P^T(i) has just been read from: the scores run two
+            // iterations ahead of the product that consumes their probabilities.
+            if (ok && n_it > 0) ok = issue_s(0, 0, true);
+            if (ok && n_it > 1) ok = issue_s(1, 1, true);
+            for (int it = 0; it < n_it && ok; ++it) {
+                const int dsl = it & 1;
+                const uint64_t dDOm = smem_desc_sw128(smem_u32(dsl ? sV : sdO), BOX64_BYTES, 1024);      // dO as MN-major B operand, all boxes
+                ok = mbar_wait(&do_full[dsl], (it >> 1) & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it));
                 if (!ok) break;
-            }
-            ok = mbar_wait(ds_ready, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it));
-            if (!ok) break;
-            tc_fence_after_sync();
-            if (elect_one()) {                     // dK[:, half] += dS^T Q[:, half]
-                const uint64_t dQm = smem_desc_sw128(smem_u32(sQ + sl * TILE64_BYTES + half * 2 * BOX64_BYTES), BOX64_BYTES, 1024);
-                if (cols_k > 0) {
+                ok = mbar_wait(&p_ready[it & 1], (it >> 1) & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it));
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (elect_one()) {                 // dV += P^T dO   (16 query rows per instruction)
 #pragma unroll
                     for (int k = 0; k < WIDE_N / 16; ++k)
-                        umma_ts(tmem_u + 256, tmem_u + 64 + k * 8, desc_advance(dQm, k * 2048), IDESC_GK, (it > 0 || k > 0) ? 1u : 0u);
+                        umma_ts(tmem_u + 128, tmem_u + (it & 1) * WIDE_N + k * 8, desc_advance(dDOm, k * 2048), IDESC_G, (it > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(&do_empty[dsl]);
+                    if (it == n_it - 1) umma_commit(final_bar);
                 }
-                umma_commit(&q_empty[sl]);
-                if (it == n_it - 1) umma_commit(final_bar);
+                __syncwarp();
+                if (it + 2 < n_it) ok = issue_s(it + 2, it & 1, true);
             }
-            __syncwarp();
-            if (it + 1 < n_it) ok = issue_dp(it + 1);     // overwrites dS^T(it): ordered behind dK(it)
+        } else {
+            // Per iteration: S(i+1) as soon as the compute warps hold S(i) in registers, dK(i), dP(i+1).
+            auto issue_dp = [&](int it) -> bool {      // dP^T = V dO^T over all columns; dO's slot is free once it has completed
+                if (!mbar_wait(&do_full[0], it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it))) return false;
+                tc_fence_after_sync();
+                if (elect_one()) {
+                    const uint64_t dDOs = smem_desc_sw128(smem_u32(sdO), 16, 1024);
+#pragma unroll
+                    for (int k = 0; k < WIDE_D / 16; ++k)
+                        if (k < kdv)
+                            umma_ss(tmem_u + 64, desc_advance(dV0, (k / 4) * BOX128_BYTES + (k % 4) * 32),
+                                    desc_advance(dDOs, (k / 4) * BOX64_BYTES + (k % 4) * 32), IDESC_S, k > 0 ? 1u : 0u);
+                    umma_commit(dp_full);
+                    umma_commit(&do_empty[0]);
+                }
+                __syncwarp();
+                return true;
+            };
+            if (ok && n_it > 0) ok = issue_s(0, 0, false);
+            if (ok && n_it > 0) ok = issue_dp(0);
+            for (int it = 0; it < n_it && ok; ++it) {
+                const int sl = it & 1;
+                ok = mbar_wait(p_ready, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it));
+                if (!ok) break;
+                if (it + 1 < n_it) {
+                    ok = issue_s(it + 1, 0, false);    // S(i) sits in the compute warps' registers: its columns are free
+                    if (!ok) break;
+                }
+                ok = mbar_wait(ds_ready, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it));
+                if (!ok) break;
+                tc_fence_after_sync();
+                if (elect_one()) {                     // dK += dS^T Q   (Q read MN-major, all boxes)
+                    const uint64_t dQm = smem_desc_sw128(smem_u32(sQ + sl * TILE64_BYTES), BOX64_BYTES, 1024);
+#pragma unroll
+                    for (int k = 0; k < WIDE_N / 16; ++k)
+                        umma_ts(tmem_u + 128, tmem_u + 64 + k * 8, desc_advance(dQm, k * 2048), IDESC_G, (it > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(&q_empty[sl]);
+                    if (it == n_it - 1) umma_commit(final_bar);
+                }
+                __syncwarp();
+                if (it + 1 < n_it) ok = issue_dp(it + 1);     // overwrites dS^T(i): ordered behind dK(i)
+            }
         }
     } else if (warp >= 4) {
         // compute: P^T, dS^T (fragment-shaped tensor-memory accesses, see vt_ptx.cuh); epilogue
@@ -272,7 +299,6 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         const int r = quad * 32 + lane;            // key row inside the tile (TMEM lane)
         const int kv = k0 + r;
         const uint32_t lane_addr = static_cast<uint32_t>(quad * 32) << 16;
-        const uint32_t tS = tmem_base + lane_addr;
         const uint32_t tDP = tmem_base + lane_addr + 64;
         const float2 c2 = make_float2(p.scale_log2e, p.scale_log2e);
         const int cq = 2 * (lane & 3);
@@ -283,9 +309,11 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             const int q0 = (qt_start + qi) * WIDE_N;
             const int rsl = it % RS;
             const float *rows = s_rows + rsl * (2 * WIDE_N);
+            const int buf = is_dv ? (it & 1) : 0;
+            const uint32_t tS = tmem_base + lane_addr + buf * WIDE_N;
             ok = mbar_wait(&rows_full[rsl], (it / RS) & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_SOFTMAX, it));
             if (!ok) break;
-            ok = mbar_wait(s_full, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_SOFTMAX, it));
+            ok = mbar_wait(&s_full[buf], (is_dv ? (it >> 1) : it) & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_SOFTMAX, it));
             if (!ok) break;
             tc_fence_after_sync();
             const bool diag = CAUSAL && (q0 + off < k0 + TILE - 1);
@@ -297,6 +325,10 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
             for (int h = 0; h < 2; ++h) tmem_ld_frag64(tS + (static_cast<uint32_t>(h * 16) << 16), sv[h]);
             tmem_wait_ld();
+            if (!is_dv) {                          // the scores are in registers: the next ones may overwrite their columns
+                tc_fence_before_sync();
+                mbar_arrive(p_ready);
+            }
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 uint32_t pp[16];
@@ -316,47 +348,48 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         pp[2 * g + rr] = pack16<F16>(e.x, e.y);
                     }
                 }
-                tmem_st_frag32(tS + (static_cast<uint32_t>(h * 16) << 16), pp);
+                if (is_dv) tmem_st_frag32(tS + (static_cast<uint32_t>(h * 16) << 16), pp);
             }
-            tmem_wait_st();
-            tc_fence_before_sync();
-            mbar_arrive(p_ready);
+            if (is_dv) {
+                tmem_wait_st();
+                tc_fence_before_sync();
+                mbar_arrive(&p_ready[buf]);
+            } else {
 #pragma unroll
-            for (int g = 0; g < 8; ++g) nl[g] = *reinterpret_cast<const float2 *>(&rows[WIDE_N + 8 * g + cq]);   // now -delta
-            ok = mbar_wait(dp_full, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_SOFTMAX, it));
-            if (!ok) break;
-            tc_fence_after_sync();
+                for (int g = 0; g < 8; ++g) nl[g] = *reinterpret_cast<const float2 *>(&rows[WIDE_N + 8 * g + cq]);   // now -delta
+                ok = mbar_wait(dp_full, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_SOFTMAX, it));
+                if (!ok) break;
+                tc_fence_after_sync();
 #pragma unroll
-            for (int h = 0; h < 2; ++h) tmem_ld_frag64(tDP + (static_cast<uint32_t>(h * 16) << 16), sv[h]);
-            tmem_wait_ld();
+                for (int h = 0; h < 2; ++h) tmem_ld_frag64(tDP + (static_cast<uint32_t>(h * 16) << 16), sv[h]);
+                tmem_wait_ld();
 #pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                uint32_t dd[16];
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t dd[16];
 #pragma unroll
-                for (int g = 0; g < 8; ++g) {
+                    for (int g = 0; g < 8; ++g) {
 #pragma unroll
-                    for (int rr = 0; rr < 2; ++rr) {
-                        const float2 df = __fadd2_rn(make_float2(__uint_as_float(sv[h][4 * g + 2 * rr]), __uint_as_float(sv[h][4 * g + 2 * rr + 1])), nl[g]);
-                        const float2 ds = __fmul2_rn(pr[h][g][rr], df);
-                        dd[2 * g + rr] = pack16<F16>(ds.x, ds.y);
+                        for (int rr = 0; rr < 2; ++rr) {
+                            const float2 df = __fadd2_rn(make_float2(__uint_as_float(sv[h][4 * g + 2 * rr]), __uint_as_float(sv[h][4 * g + 2 * rr + 1])), nl[g]);
+                            const float2 ds = __fmul2_rn(pr[h][g][rr], df);
+                            dd[2 * g + rr] = pack16<F16>(ds.x, ds.y);
+                        }
                     }
+                    tmem_st_frag32(tDP + (static_cast<uint32_t>(h * 16) << 16), dd);
                 }
-                tmem_st_frag32(tDP + (static_cast<uint32_t>(h * 16) << 16), dd);
+                tmem_wait_st();
+                tc_fence_before_sync();
+                mbar_arrive(ds_ready);
             }
-            tmem_wait_st();
-            tc_fence_before_sync();
-            mbar_arrive(ds_ready);
             __syncwarp();
             if (lane == 0) mbar_arrive(&rows_empty[rsl]);
         }
-        // epilogue: this block's column half of dV, then of dK
-        const size_t row_v = (static_cast<size_t>(bh_kv) * p.Sk + kv) * dv_w + half * TILE;
-        const size_t row_k = (static_cast<size_t>(bh_kv) * p.Sk + kv) * p.d + half * TILE;
+        // epilogue: this block's tensor, all its columns
+        __nv_bfloat16 *out = is_dv ? p.dv : p.dk;
+        const size_t row_o = (static_cast<size_t>(bh_kv) * p.Sk + kv) * out_w;
         if (n_it == 0) {
-            if (kv < Sk) {
-                for (int i = 0; i < cols_v / 8; ++i) reinterpret_cast<uint4 *>(p.dv + row_v)[i] = make_uint4(0, 0, 0, 0);
-                for (int i = 0; i < cols_k / 8; ++i) reinterpret_cast<uint4 *>(p.dk + row_k)[i] = make_uint4(0, 0, 0, 0);
-            }
+            if (kv < Sk)
+                for (int i = 0; i < out_w / 8; ++i) reinterpret_cast<uint4 *>(out + row_o)[i] = make_uint4(0, 0, 0, 0);
         } else {
             if (ok) ok = mbar_wait(final_bar, 0, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_EPILOGUE, 0));
             if (ok) {
@@ -364,21 +397,16 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 uint8_t *scratch = sQ + (warp - 4) * STORE_SCRATCH_BYTES;     // every product has completed: the Q slots are free
                 const int row0 = k0 + quad * 32;
                 const int rows_valid = min(32, Sk - row0);
+                const size_t stride = static_cast<size_t>(out_w);
+                __nv_bfloat16 *warp_dst = out + row_o - static_cast<size_t>(lane) * stride;
+                const float mul = is_dv ? 1.0f : p.scale;
 #pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                    const size_t stride = static_cast<size_t>(t == 0 ? dv_w : p.d);
-                    const int cols_out = (t == 0) ? cols_v : cols_k;
-                    __nv_bfloat16 *warp_dst = (t == 0 ? p.dv + row_v : p.dk + row_k) - static_cast<size_t>(lane) * stride;
-                    const uint32_t tSrc = tmem_base + lane_addr + 128 + t * 128;
-                    const float mul = (t == 0) ? 1.0f : p.scale;
-                    if (cols_out <= 0) continue;                       // this half holds no column of the tensor (block-uniform)
-#pragma unroll
-                    for (int c = 0; c < TILE / 32; ++c) {
-                        uint32_t v[32];
-                        tmem_ld32(tSrc + c * 32, v);
-                        tmem_wait_ld();
-                        store_rows16<F16>(warp_dst + c * 32, stride, v, mul, rows_valid, scratch, lane, cols_out - c * 32);
-                    }
+                for (int c = 0; c < WIDE_D / 32; ++c) {
+                    if (c * 32 >= out_w) break;                            // block-uniform
+                    uint32_t v[32];
+                    tmem_ld32(tmem_base + lane_addr + 128 + c * 32, v);
+                    tmem_wait_ld();
+                    store_rows16<F16>(warp_dst + c * 32, stride, v, mul, rows_valid, scratch, lane, out_w - c * 32);
                 }
             }
         }
@@ -689,8 +717,7 @@ static int launch_wide(const CUtensorMap &q64, const CUtensorMap &do64, const CU
     if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_delta_kernel launch");
 
     prm.n_tiles = (prm.Sk + TILE - 1) / TILE;
-    const int widest = prm.d > prm.d_v ? prm.d : prm.d_v;
-    const dim3 grid_kv(static_cast<unsigned>(prm.n_tiles * B * prm.Hkv), widest > TILE ? 2 : 1);      // one pass per 128 columns of dK / dV
+    const dim3 grid_kv(static_cast<unsigned>(prm.n_tiles * B * prm.Hkv), 2);      // a dK block and a dV block per key tile
     bwd_dkdv_wide_kernel<CAUSAL, F16><<<grid_kv, WIDE_THREADS, DkdvWideSmem::BYTES, stream>>>(q64, k128, v128, do64, prm);
     if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_dkdv_wide_kernel launch");
 

@@ -23,7 +23,7 @@ constexpr unsigned long long DEFAULT_WAIT_LIMIT_NS = 2000000000ull;   // 2 s per
 // built for 64, 128 and (forward only) 256 columns; any other dimension runs in the next larger one: the TMA boxes read
 // the columns past the row's end as zero, which adds nothing to S = Q K^T, and the epilogues store only the real columns.
 constexpr int MAX_HEAD_DIM = 128;          // packed and split-KV entry points, the one-pass kernels
-constexpr int MAX_HEAD_DIM_FWD = 256;      // batched forward and backward (the backward above 128 columns in two column halves)
+constexpr int MAX_HEAD_DIM_FWD = 256;      // batched forward and backward (the backward above 128 columns: bwd_wide.cu)
 inline bool head_dim_ok(int D, int max_d = MAX_HEAD_DIM) { return D >= 8 && D <= max_d && D % 8 == 0; }
 inline int padded_head_dim(int D) { return D <= 64 ? 64 : (D <= 128 ? 128 : 256); }
 

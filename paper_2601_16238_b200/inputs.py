@@ -65,7 +65,7 @@ CONFIGS = {
     "gqa_long": AttnConfig("gqa_long", 5, 1, 32, 8, 16384, 16384, 128, True, True),
     # a long D=64 shape (not a graded config): the exponential unit, not the tensor core, bounds it
     "d64_s4096_nc": AttnConfig("d64_s4096_nc", 7, 4, 16, 16, 4096, 4096, 64, False, True),
-    # a long D=256 shape (not a graded config): the forward with 256 columns, the backward in two column halves
+    # a long D=256 shape (not a graded config): the forward with 256 columns, the backward's kernels for 128 < D <= 256
     "d256_s4096_nc": AttnConfig("d256_s4096_nc", 8, 4, 8, 8, 4096, 4096, 256, False, True),
     # low-occupancy shapes for the split-KV forward: one decoded token against a long cache, and a prefill chunk at the
     # end of a long context (bottom-right aligned mask); forward only

@@ -1,5 +1,5 @@
 """GPU: the backward for head dimensions above 128 (up to 256): Delta, a dK/dV kernel that keeps 128 keys x 256 columns
-stationary and walks the queries 64 at a time (twice: one half of the output columns per pass), and a dQ kernel that
+stationary and walks the queries 64 at a time (in two blocks: one accumulates dK, the other dV), and a dQ kernel that
 keeps 128 queries stationary and walks the keys 64 at a time - against the fp64 oracle, element by element."""
 import numpy as np
 import pytest
@@ -15,7 +15,7 @@ SHAPES = [
     (1, 1, 1, 128, 128, 256, 0),
     (1, 2, 2, 64, 64, 256, 1),
     (1, 2, 1, 200, 333, 256, 0),          # ragged ends, two heads per KV head
-    (2, 4, 2, 300, 300, 192, 1),          # the other common size: the second column half holds 64 columns
+    (2, 4, 2, 300, 300, 192, 1),          # the other common size: 192 = 3 boxes of 64 columns
     (1, 2, 2, 257, 129, 136, 1),          # eight columns in the second half; top-left mask with Sq > Sk
     (1, 2, 1, 190, 450, 256, 2),          # bottom-right aligned mask
     (1, 2, 2, 450, 190, 200, 2),          # fewer keys than queries: leading rows see nothing
