@@ -6,7 +6,7 @@ import os
 import numpy as np
 import pytest
 
-from helpers import check_fwd, check_grad, dev, host
+from helpers import TOL_GRAD, TOL_LSE, TOL_O, check_fwd, check_grad, dev, host
 from oracle import attn_oracle as orc
 from paper_2601_16238_b200.inputs import CONFIGS, AttnConfig, make_inputs
 
@@ -140,6 +140,24 @@ def test_gqa_causal_d128_multi_tile_full_parity(vt):
     """Same structure as the long-context config (GQA 4:1, causal, D = 128) at a size the oracle
     finishes in seconds, element by element for all of dQ, dK, dV."""
     full_parity(vt, CONFIGS["gqa_long"].with_(Sq=640, Sk=640), "gqa 640")
+
+
+def test_d64_workload_full_length_heads(vt):
+    """Two full-length heads of the benchmark's 64-column workload (4096 queries and keys): forward and backward, every
+    element against the oracle."""
+    import torch
+    cfg = CONFIGS["d64_s4096_nc"].with_(B=1, Hq=2, Hkv=2)
+    q, k, v, d_o = make_inputs(cfg)
+    tq, tk, tv, tdo = dev(q), dev(k), dev(v), dev(d_o)
+    o, lse = vt.vt_attn_fwd(tq, tk, tv, cfg.causal, cfg.scale)
+    grads = vt.vt_attn_bwd(tq, tk, tv, o, tdo, lse, cfg.causal, cfg.scale)
+    torch.cuda.synchronize()
+    assert vt.vt_attn_device_status()[0] == 0
+    o_ref, lse_ref = orc.attn_fwd(q, k, v, cfg.causal, cfg.scale)
+    assert np.abs(host(o) - o_ref).max() <= TOL_O
+    assert (np.abs(host(lse) - lse_ref) <= TOL_LSE * np.maximum(1.0, np.abs(lse_ref))).all()
+    for nm, a, b in zip(("dQ", "dK", "dV"), grads, orc.attn_bwd(q, k, v, d_o, cfg.causal, cfg.scale)):
+        assert np.abs(host(a) - b).max() <= TOL_GRAD * np.abs(b).max(), nm
 
 
 def test_paper_shape_reduced_batch(vt):

@@ -85,6 +85,23 @@ def test_decode_shape_at_full_size_sampled_heads(vt):
         assert (np.abs(host(lse[b:b + 1]) - lse_ref) <= TOL_LSE * np.maximum(1.0, np.abs(lse_ref))).all()
 
 
+def test_prefill_chunk_shape_at_full_size(vt):
+    """The prefill benchmark shape (512 new queries at the end of a 16384-token context, 32 query heads on 8 KV heads,
+    bottom-right mask) at full size: every row of O and LSE against the oracle, through the split-KV entry point with the
+    split count the library picks and through the plain forward."""
+    import torch
+    cfg = AttnConfig("prefill_chunk", 13, 1, 32, 8, 512, 16384, 128, 2, False)
+    q, k, v = make_inputs(cfg, with_do=False)
+    tq, tk, tv = dev(q), dev(k), dev(v)
+    o_ref, lse_ref = orc.attn_fwd(q, k, v, 2, cfg.scale)
+    for call in (lambda: vt.vt_attn_fwd_splitkv(tq, tk, tv, 2, cfg.scale), lambda: vt.vt_attn_fwd(tq, tk, tv, 2, cfg.scale)):
+        o, lse = call()
+        torch.cuda.synchronize()
+        assert vt.vt_attn_device_status()[0] == 0
+        assert np.abs(host(o) - o_ref).max() <= TOL_O
+        assert (np.abs(host(lse) - lse_ref) <= TOL_LSE * np.maximum(1.0, np.abs(lse_ref))).all()
+
+
 PACKED_CASES = [
     # Hq, Hkv, D, causal, query lengths, key lengths, n_splits
     (8, 2, 128, 2, [1, 1, 1, 1, 1], [1000, 37, 2049, 513, 1], 0),            # decoding against caches of different lengths; heads share a tile
