@@ -52,6 +52,20 @@ __device__ __forceinline__ uint4 pack8(const float (&f)[8])
     return make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
 }
 
+// The same eight values as four pairs: the norm kernels do their arithmetic two elements per instruction (fma / add / mul
+// .f32x2, each half rounded like the scalar instruction), which is what keeps them off the issue-slot limit.
+__device__ __forceinline__ void unpack8(const uint4 &u, float2 (&f)[4])
+{
+    f[0] = unpack16<false>(u.x); f[1] = unpack16<false>(u.y); f[2] = unpack16<false>(u.z); f[3] = unpack16<false>(u.w);
+}
+
+__device__ __forceinline__ uint4 pack8(const float2 (&f)[4])
+{
+    return make_uint4(pack_bf16(f[0].x, f[0].y), pack_bf16(f[1].x, f[1].y), pack_bf16(f[2].x, f[2].y), pack_bf16(f[3].x, f[3].y));
+}
+
+__device__ __forceinline__ float2 splat2(float v) { return make_float2(v, v); }
+
 // ----------------------------------------------------------------------------------------------
 // RMSNorm forward.  VPT: 16-byte vectors per thread (a row has nvec = cols / 8 of them, vector v of thread t is
 // number v * T + t).
@@ -68,25 +82,27 @@ __global__ void __launch_bounds__(T) rmsnorm_fwd_kernel(const uint4 *__restrict_
         uint4 xv[VPT];
 #pragma unroll
         for (int v = 0; v < VPT; ++v) xv[v] = (v * nt + tid < nvec) ? xr[v * nt + tid] : make_uint4(0, 0, 0, 0);
-        float ss[1] = {0.0f};
+        float2 ss2 = make_float2(0.0f, 0.0f);
 #pragma unroll
         for (int v = 0; v < VPT; ++v) {
-            float f[8];
+            float2 f[4];
             unpack8(xv[v], f);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) ss[0] = fmaf(f[e], f[e], ss[0]);
+            for (int e = 0; e < 4; ++e) ss2 = __ffma2_rn(f[e], f[e], ss2);
         }
+        float ss[1] = {ss2.x + ss2.y};
         block_sum<1>(ss, red, turn);
         const float r = 1.0f / sqrtf(ss[0] * inv_cols + eps);
+        const float2 r2 = splat2(r);
         uint4 *yr = y + row * nvec;
 #pragma unroll
         for (int v = 0; v < VPT; ++v) {
             if (v * nt + tid < nvec) {
-                float f[8], g[8];
+                float2 f[4], g[4];
                 unpack8(xv[v], f);
                 unpack8(__ldg(w + v * nt + tid), g);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) f[e] = f[e] * r * g[e];
+                for (int e = 0; e < 4; ++e) f[e] = __fmul2_rn(__fmul2_rn(f[e], r2), g[e]);
                 yr[v * nt + tid] = pack8(f);
             }
         }
@@ -110,39 +126,45 @@ __global__ void __launch_bounds__(T) layernorm_fwd_kernel(const uint4 *__restric
         uint4 xv[VPT];
 #pragma unroll
         for (int v = 0; v < VPT; ++v) xv[v] = (v * nt + tid < nvec) ? xr[v * nt + tid] : make_uint4(0, 0, 0, 0);
-        float s[1] = {0.0f};
+        float2 s2 = make_float2(0.0f, 0.0f);
 #pragma unroll
         for (int v = 0; v < VPT; ++v) {
-            float f[8];
+            float2 f[4];
             unpack8(xv[v], f);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) s[0] += f[e];
+            for (int e = 0; e < 4; ++e) s2 = __fadd2_rn(s2, f[e]);
         }
+        float s[1] = {s2.x + s2.y};
         block_sum<1>(s, red, turn);
         const float mu = s[0] * inv_cols;
-        float q[1] = {0.0f};
+        const float2 nmu2 = splat2(-mu);
+        float2 q2 = make_float2(0.0f, 0.0f);
 #pragma unroll
         for (int v = 0; v < VPT; ++v) {
             if (v * nt + tid < nvec) {                 // (the padding vectors must not add mu^2)
-                float f[8];
+                float2 f[4];
                 unpack8(xv[v], f);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) q[0] = fmaf(f[e] - mu, f[e] - mu, q[0]);
+                for (int e = 0; e < 4; ++e) {
+                    const float2 d = __fadd2_rn(f[e], nmu2);
+                    q2 = __ffma2_rn(d, d, q2);
+                }
             }
         }
+        float q[1] = {q2.x + q2.y};
         block_sum<1>(q, red, turn);
         const float r = 1.0f / sqrtf(q[0] * inv_cols + eps);
-        const float nmr = -mu * r;
+        const float2 r2 = splat2(r), nmr2 = splat2(-mu * r);
         uint4 *yr = y + row * nvec;
 #pragma unroll
         for (int v = 0; v < VPT; ++v) {
             if (v * nt + tid < nvec) {
-                float f[8], g[8], h[8];
+                float2 f[4], g[4], h[4];
                 unpack8(xv[v], f);
                 unpack8(__ldg(w + v * nt + tid), g);
                 unpack8(__ldg(b + v * nt + tid), h);
 #pragma unroll
-                for (int e = 0; e < 8; ++e) f[e] = fmaf(fmaf(f[e], r, nmr), g[e], h[e]);
+                for (int e = 0; e < 4; ++e) f[e] = __ffma2_rn(__ffma2_rn(f[e], r2, nmr2), g[e], h[e]);
                 yr[v * nt + tid] = pack8(f);
             }
         }
@@ -172,11 +194,11 @@ __global__ void __launch_bounds__(1024 / VPT) layernorm_bwd_kernel(const uint4 *
     __shared__ float red[128];
     uint32_t turn = 0;
     const int tid = threadIdx.x, nt = blockDim.x;
-    float aw[VPT][8], ab[VPT][8];
+    float2 aw[VPT][4], ab[VPT][4];
 #pragma unroll
     for (int v = 0; v < VPT; ++v)
 #pragma unroll
-        for (int e = 0; e < 8; ++e) aw[v][e] = ab[v][e] = 0.0f;
+        for (int e = 0; e < 4; ++e) aw[v][e] = ab[v][e] = make_float2(0.0f, 0.0f);
     const uint4 zero = make_uint4(0, 0, 0, 0);
     long long row = blockIdx.x;
     uint4 xv[VPT], gv[VPT];
@@ -209,34 +231,35 @@ __global__ void __launch_bounds__(1024 / VPT) layernorm_bwd_kernel(const uint4 *
             mun = RMS ? 0.0f : mean[next];
             rn = rstd[next];
         }
-        float xh[VPT][8], g[VPT][8];
-        float s[2] = {0.0f, 0.0f};          // sum_j g, sum_j g * xh   (vectors past the row's end hold dy = 0, w = 0: they add nothing)
-        const float nmr = -mu * r;
+        float2 xh[VPT][4], g[VPT][4];
+        float2 s0 = make_float2(0.0f, 0.0f), s1 = make_float2(0.0f, 0.0f);   // sum_j g, sum_j g * xh   (vectors past the row's end hold dy = 0, w = 0: they add nothing)
+        const float2 r2 = splat2(r), nmr2 = splat2(-mu * r);
 #pragma unroll
         for (int v = 0; v < VPT; ++v) {
-            float f[8], d[8];
+            float2 f[4], d[4];
             unpack8(xv[v], f);
             unpack8(gv[v], d);
             unpack8((v * nt + tid < nvec) ? __ldg(w + v * nt + tid) : zero, g[v]);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) {
-                xh[v][e] = fmaf(f[e], r, nmr);
-                g[v][e] *= d[e];
-                s[0] += g[v][e];
-                s[1] = fmaf(g[v][e], xh[v][e], s[1]);
-                aw[v][e] = fmaf(d[e], xh[v][e], aw[v][e]);
-                if (!RMS) ab[v][e] += d[e];
+            for (int e = 0; e < 4; ++e) {
+                xh[v][e] = __ffma2_rn(f[e], r2, nmr2);
+                g[v][e] = __fmul2_rn(g[v][e], d[e]);
+                s0 = __fadd2_rn(s0, g[v][e]);
+                s1 = __ffma2_rn(g[v][e], xh[v][e], s1);
+                aw[v][e] = __ffma2_rn(d[e], xh[v][e], aw[v][e]);
+                if (!RMS) ab[v][e] = __fadd2_rn(ab[v][e], d[e]);
             }
         }
+        float s[2] = {s0.x + s0.y, s1.x + s1.y};
         block_sum<2>(s, red, turn);
         const float m1 = RMS ? 0.0f : s[0] * inv_cols, m2 = s[1] * inv_cols;
-        const float c1 = -r * m1, c2 = -r * m2;
+        const float2 c1 = splat2(-r * m1), c2 = splat2(-r * m2);
 #pragma unroll
         for (int v = 0; v < VPT; ++v)
             if (v * nt + tid < nvec) {
-                float f[8];
+                float2 f[4];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) f[e] = fmaf(xh[v][e], c2, fmaf(g[v][e], r, c1));
+                for (int e = 0; e < 4; ++e) f[e] = __ffma2_rn(xh[v][e], c2, __ffma2_rn(g[v][e], r2, c1));
                 dx[row * nvec + v * nt + tid] = pack8(f);
             }
 #pragma unroll
@@ -254,11 +277,11 @@ __global__ void __launch_bounds__(1024 / VPT) layernorm_bwd_kernel(const uint4 *
             const size_t c = static_cast<size_t>(v * nt + tid) * 8;
             float *pw = part + static_cast<size_t>(blockIdx.x) * cols + c;
             float *pb = part + (static_cast<size_t>(gridDim.x) + blockIdx.x) * cols + c;
-            *reinterpret_cast<float4 *>(pw) = make_float4(aw[v][0], aw[v][1], aw[v][2], aw[v][3]);
-            *reinterpret_cast<float4 *>(pw + 4) = make_float4(aw[v][4], aw[v][5], aw[v][6], aw[v][7]);
+            *reinterpret_cast<float4 *>(pw) = make_float4(aw[v][0].x, aw[v][0].y, aw[v][1].x, aw[v][1].y);
+            *reinterpret_cast<float4 *>(pw + 4) = make_float4(aw[v][2].x, aw[v][2].y, aw[v][3].x, aw[v][3].y);
             if (!RMS) {
-                *reinterpret_cast<float4 *>(pb) = make_float4(ab[v][0], ab[v][1], ab[v][2], ab[v][3]);
-                *reinterpret_cast<float4 *>(pb + 4) = make_float4(ab[v][4], ab[v][5], ab[v][6], ab[v][7]);
+                *reinterpret_cast<float4 *>(pb) = make_float4(ab[v][0].x, ab[v][0].y, ab[v][1].x, ab[v][1].y);
+                *reinterpret_cast<float4 *>(pb + 4) = make_float4(ab[v][2].x, ab[v][2].y, ab[v][3].x, ab[v][3].y);
             }
         }
 }
