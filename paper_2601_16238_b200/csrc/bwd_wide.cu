@@ -8,7 +8,8 @@
 //       columns together would fill tensor memory).  K stays in shared memory; the query heads of the group are walked
 //       64 queries at a time (Q in two slots) and S^T = K Q^T contracts over all columns in both blocks.  The dK block also
 //       holds V, forms dP^T = V dO^T and dS^T and accumulates dK += dS^T Q (N = 256); the dV block only needs P^T and
-//       accumulates dV += P^T dO, with two score buffers and two dO slots.
+//       accumulates dV += P^T dO, with two score buffers and two dO slots.  Tensors of at most 192 columns leave room
+//       for both accumulators: then one block per key tile does both and forms the scores once.
 //   bwd_dq_wide_kernel   : one block per (batch, query head, 128-query tile).  Q and dO stay in shared memory, K (two
 //       slots) and V (one slot) stream by in tiles of 64 keys; dQ (256 columns) is accumulated in tensor memory.
 //
@@ -43,6 +44,7 @@ struct DkdvWideSmem {
     static constexpr int BYTES = OFF_BAR + 256;                      // no alignment slack: the kernel checks the base address
     // TMEM columns.  dK block: S^T [0,64), dP^T [64,128) (dS^T, 16-bit, over its first 32), dK [128,384).
     // dV block: two S^T buffers [0,64), [64,128) (P^T, 16-bit, over the first 32 of each), dV [128,384).
+    // Block for both (widths <= 192): S^T [0,64) (P^T over its first 32), dP^T [64,128), dV [128,320), dK [320,512).
     static constexpr int TMEM_COLS = 512;
 };
 
@@ -89,7 +91,12 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
         return;
     }
 
-    const bool is_dv = blockIdx.y != 0;                   // block-uniform: the longer dK blocks come first in the launch
+    // Block-uniform role.  Two blocks per key tile (gridDim.y = 2): 0 accumulates dK, 1 accumulates dV; the longer dK blocks
+    // come first in the launch.  One block per key tile (gridDim.y = 1, tensors of at most 192 columns, whose two
+    // accumulators fit beside S^T and dP^T): 2, both - the scores are formed once.
+    const int role = (gridDim.y == 1) ? 2 : static_cast<int>(blockIdx.y);
+    const bool is_dv = role == 1;                         // the dV-only block: two score buffers, two dO slots, no V, no dP
+    const bool has_dv = role != 0, has_dk = role != 1;
     const int bh_kv = blockIdx.x / p.n_tiles;
     const int kt = blockIdx.x % p.n_tiles;
     const int b = bh_kv / p.Hkv;
@@ -102,7 +109,8 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
     const int n_qi = n_qt - qt_start;
     const int n_it = n_qi * p.G;
     const int dv_w = p.d_v > 0 ? p.d_v : p.d;             // width of V, dO, dV (Q, K, dK: p.d)
-    const int out_w = is_dv ? dv_w : p.d;                 // columns of this block's output tensor
+    const int out_w = is_dv ? dv_w : p.d;                 // columns of this block's (first) output tensor: dV for role 1, else dK
+    const uint32_t acc_k = 128 + (role == 2 ? 192 : 0);   // tensor-memory column of the dK accumulator (dV: always 128)
     const int kd = (p.d + 15) >> 4;                       // 16-column contraction steps of S^T = K Q^T that hold data
     const int kdv = (dv_w + 15) >> 4;                     // of dP^T = V dO^T
 
@@ -251,8 +259,12 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 if (it + 2 < n_it) ok = issue_s(it + 2, it & 1, true);
             }
         } else {
-            // Per iteration: S(i+1) as soon as the compute warps hold S(i) in registers, dK(i), dP(i+1).
-            auto issue_dp = [&](int it) -> bool {      // dP^T = V dO^T over all columns; dO's slot is free once it has completed
+            // dK block, per iteration: S(i+1) as soon as the compute warps hold S(i) in registers, dK(i), dP(i+1).
+            // Block for both: dV(i) once P^T(i) is in tensor memory, S(i+1) behind it (it overwrites P^T(i)), dK(i), dP(i+1).
+            const uint32_t IDESC_GV = make_idesc(128, ((dv_w + 15) >> 4) * 16, fmt16<F16>(), fmt16<F16>(), 0, 1);
+            const uint64_t dDOm = smem_desc_sw128(smem_u32(sdO), BOX64_BYTES, 1024);      // dO as MN-major B operand of dV
+            // dP^T = V dO^T over all columns; free_do: nothing else reads this dO tile (dK block)
+            auto issue_dp = [&](int it, bool free_do) -> bool {
                 if (!mbar_wait(&do_full[0], it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it))) return false;
                 tc_fence_after_sync();
                 if (elect_one()) {
@@ -263,19 +275,30 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                             umma_ss(tmem_u + 64, desc_advance(dV0, (k / 4) * BOX128_BYTES + (k % 4) * 32),
                                     desc_advance(dDOs, (k / 4) * BOX64_BYTES + (k % 4) * 32), IDESC_S, k > 0 ? 1u : 0u);
                     umma_commit(dp_full);
-                    umma_commit(&do_empty[0]);
+                    if (free_do) umma_commit(&do_empty[0]);
                 }
                 __syncwarp();
                 return true;
             };
             if (ok && n_it > 0) ok = issue_s(0, 0, false);
-            if (ok && n_it > 0) ok = issue_dp(0);
+            if (ok && n_it > 0) ok = issue_dp(0, !has_dv);
             for (int it = 0; it < n_it && ok; ++it) {
                 const int sl = it & 1;
                 ok = mbar_wait(p_ready, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it));
                 if (!ok) break;
+                if (has_dv) {
+                    tc_fence_after_sync();
+                    if (elect_one()) {                 // dV += P^T dO   (dO was read by dP(i) before: its slot is free after this)
+#pragma unroll
+                        for (int k = 0; k < WIDE_N / 16; ++k)
+                            umma_ts(tmem_u + 128, tmem_u + k * 8, desc_advance(dDOm, k * 2048), IDESC_GV, (it > 0 || k > 0) ? 1u : 0u);
+                        umma_commit(&do_empty[0]);
+                    }
+                    __syncwarp();
+                }
                 if (it + 1 < n_it) {
-                    ok = issue_s(it + 1, 0, false);    // S(i) sits in the compute warps' registers: its columns are free
+                    // dK block: S(i) sits in the compute warps' registers, its columns are free; both: ordered behind dV(i)
+                    ok = issue_s(it + 1, 0, false);
                     if (!ok) break;
                 }
                 ok = mbar_wait(ds_ready, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_MMA, it));
@@ -285,12 +308,12 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                     const uint64_t dQm = smem_desc_sw128(smem_u32(sQ + sl * TILE64_BYTES), BOX64_BYTES, 1024);
 #pragma unroll
                     for (int k = 0; k < WIDE_N / 16; ++k)
-                        umma_ts(tmem_u + 128, tmem_u + 64 + k * 8, desc_advance(dQm, k * 2048), IDESC_G, (it > 0 || k > 0) ? 1u : 0u);
+                        umma_ts(tmem_u + acc_k, tmem_u + 64 + k * 8, desc_advance(dQm, k * 2048), IDESC_G, (it > 0 || k > 0) ? 1u : 0u);
                     umma_commit(&q_empty[sl]);
                     if (it == n_it - 1) umma_commit(final_bar);
                 }
                 __syncwarp();
-                if (it + 1 < n_it) ok = issue_dp(it + 1);     // overwrites dS^T(i): ordered behind dK(i)
+                if (it + 1 < n_it) ok = issue_dp(it + 1, !has_dv);     // overwrites dS^T(i): ordered behind dK(i)
             }
         }
     } else if (warp >= 4) {
@@ -325,7 +348,7 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
 #pragma unroll
             for (int h = 0; h < 2; ++h) tmem_ld_frag64(tS + (static_cast<uint32_t>(h * 16) << 16), sv[h]);
             tmem_wait_ld();
-            if (!is_dv) {                          // the scores are in registers: the next ones may overwrite their columns
+            if (!has_dv) {                         // dK block: the scores are in registers, the next ones may overwrite their columns
                 tc_fence_before_sync();
                 mbar_arrive(p_ready);
             }
@@ -348,13 +371,14 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                         pp[2 * g + rr] = pack16<F16>(e.x, e.y);
                     }
                 }
-                if (is_dv) tmem_st_frag32(tS + (static_cast<uint32_t>(h * 16) << 16), pp);
+                if (has_dv) tmem_st_frag32(tS + (static_cast<uint32_t>(h * 16) << 16), pp);
             }
-            if (is_dv) {
+            if (has_dv) {
                 tmem_wait_st();
                 tc_fence_before_sync();
                 mbar_arrive(&p_ready[buf]);
-            } else {
+            }
+            if (has_dk) {
 #pragma unroll
                 for (int g = 0; g < 8; ++g) nl[g] = *reinterpret_cast<const float2 *>(&rows[WIDE_N + 8 * g + cq]);   // now -delta
                 ok = mbar_wait(dp_full, it & 1, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_SOFTMAX, it));
@@ -384,12 +408,13 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
             __syncwarp();
             if (lane == 0) mbar_arrive(&rows_empty[rsl]);
         }
-        // epilogue: this block's tensor, all its columns
-        __nv_bfloat16 *out = is_dv ? p.dv : p.dk;
-        const size_t row_o = (static_cast<size_t>(bh_kv) * p.Sk + kv) * out_w;
+        // epilogue: this block's tensor(s), all their columns
+        const size_t key_row = static_cast<size_t>(bh_kv) * p.Sk + kv;
         if (n_it == 0) {
-            if (kv < Sk)
-                for (int i = 0; i < out_w / 8; ++i) reinterpret_cast<uint4 *>(out + row_o)[i] = make_uint4(0, 0, 0, 0);
+            if (kv < Sk) {
+                if (has_dv) for (int i = 0; i < dv_w / 8; ++i) reinterpret_cast<uint4 *>(p.dv + key_row * dv_w)[i] = make_uint4(0, 0, 0, 0);
+                if (has_dk) for (int i = 0; i < p.d / 8; ++i) reinterpret_cast<uint4 *>(p.dk + key_row * p.d)[i] = make_uint4(0, 0, 0, 0);
+            }
         } else {
             if (ok) ok = mbar_wait(final_bar, 0, abort_flag, p.guard, status_word(DKDV_WIDE_KERNEL_ID, ROLE_EPILOGUE, 0));
             if (ok) {
@@ -397,16 +422,22 @@ bwd_dkdv_wide_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_cons
                 uint8_t *scratch = sQ + (warp - 4) * STORE_SCRATCH_BYTES;     // every product has completed: the Q slots are free
                 const int row0 = k0 + quad * 32;
                 const int rows_valid = min(32, Sk - row0);
-                const size_t stride = static_cast<size_t>(out_w);
-                __nv_bfloat16 *warp_dst = out + row_o - static_cast<size_t>(lane) * stride;
-                const float mul = is_dv ? 1.0f : p.scale;
 #pragma unroll
-                for (int c = 0; c < WIDE_D / 32; ++c) {
-                    if (c * 32 >= out_w) break;                            // block-uniform
-                    uint32_t v[32];
-                    tmem_ld32(tmem_base + lane_addr + 128 + c * 32, v);
-                    tmem_wait_ld();
-                    store_rows16<F16>(warp_dst + c * 32, stride, v, mul, rows_valid, scratch, lane, out_w - c * 32);
+                for (int t = 0; t < 2; ++t) {                                  // t = 0: dV, 1: dK
+                    if (t == 0 ? !has_dv : !has_dk) continue;                  // block-uniform
+                    const int w_out = (t == 0) ? dv_w : p.d;
+                    const size_t stride = static_cast<size_t>(w_out);
+                    __nv_bfloat16 *warp_dst = (t == 0 ? p.dv : p.dk) + key_row * stride - static_cast<size_t>(lane) * stride;
+                    const uint32_t tSrc = tmem_base + lane_addr + (t == 0 ? 128u : acc_k);
+                    const float mul = (t == 0) ? 1.0f : p.scale;
+#pragma unroll
+                    for (int c = 0; c < WIDE_D / 32; ++c) {
+                        if (c * 32 >= w_out) break;                        // block-uniform
+                        uint32_t v[32];
+                        tmem_ld32(tSrc + c * 32, v);
+                        tmem_wait_ld();
+                        store_rows16<F16>(warp_dst + c * 32, stride, v, mul, rows_valid, scratch, lane, w_out - c * 32);
+                    }
                 }
             }
         }
@@ -717,7 +748,10 @@ static int launch_wide(const CUtensorMap &q64, const CUtensorMap &do64, const CU
     if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_delta_kernel launch");
 
     prm.n_tiles = (prm.Sk + TILE - 1) / TILE;
-    const dim3 grid_kv(static_cast<unsigned>(prm.n_tiles * B * prm.Hkv), 2);      // a dK block and a dV block per key tile
+    // a dK block and a dV block per key tile; one block for both when the two accumulators (at most 192 columns each) fit
+    // beside S^T and dP^T in tensor memory
+    const int dv_cols = prm.d_v > 0 ? prm.d_v : prm.d;
+    const dim3 grid_kv(static_cast<unsigned>(prm.n_tiles * B * prm.Hkv), (prm.d <= 192 && dv_cols <= 192) ? 1 : 2);
     bwd_dkdv_wide_kernel<CAUSAL, F16><<<grid_kv, WIDE_THREADS, DkdvWideSmem::BYTES, stream>>>(q64, k128, v128, do64, prm);
     if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "bwd_dkdv_wide_kernel launch");
 
